@@ -1,0 +1,159 @@
+/*
+ * def.h -- C boundary of the B200 (sm_100a) DEF / DEF-A / EF step library.
+ *
+ * One optimizer step of distributed momentum SGD with random block-wise gradient
+ * sparsification (RBGS) under error feedback, from "Detached Error Feedback for
+ * Distributed SGD with Random Sparsification": Algorithm 1 lines 7-10 with the
+ * momentum substitution of Eq. 10, for W simulated workers (the paper's K) held as
+ * the rows of [W, d] fp32 tensors on one GPU.  Per step and per worker w:
+ *
+ *     m'[w,j] = mu * m[w,j] + g[w,j]                          (Eq. 10)
+ *     p[w,j]  = eta * m'[w,j] + e[w,j]                        (Eq. 10; Algorithm 1 line 7 when mu = 0)
+ *     C(p)    = p on the k block coordinates {(s+i) mod d}, 0 elsewhere   (Section 1, RBGS)
+ *     e'[w,j] = p[w,j] - C(p)[w,j]                            (Algorithm 1 line 8)
+ *     x[j]   -= (1/W) * sum_w C(p)[w,j]                       (Algorithm 1 lines 9-10)
+ *
+ * The block start s is drawn once per step, the same for every worker (Section 1:
+ * all workers hold the same seed), by a counter-based Philox4x32-10 generator keyed
+ * by (seed, step).  The sum over workers stands in for the ring-allreduce of line 9;
+ * it runs over w = 0..W-1 in that order in fp32, followed by an IEEE division by W.
+ * Every product-and-add above is one fused multiply-add (one rounding).
+ *
+ * EF, DEF and DEF-A run the same step: they differ in where the caller evaluates
+ * the gradient (Algorithm 1 line 6: at x_t - lambda e_{k,t}, lambda = 0 for EF) and
+ * in the model that is returned after training (Algorithm 1's output line).
+ *
+ * Conventions
+ *   - All tensors are fp32, row-major; [W, d] tensors are contiguous with row stride d
+ *     unless a call takes an explicit row stride `ld` (in floats).
+ *   - Pointers are DEVICE pointers on the current CUDA device unless the parameter is
+ *     called *_host.  The caller owns every tensor; the library keeps no reference to
+ *     them after the work it enqueued has run.
+ *   - Calls that take device pointers only enqueue work on the context's stream
+ *     (def_set_stream; default: the legacy default stream).  They do not synchronise
+ *     and they allocate nothing.
+ *   - Every function returns DEF_OK (0) or a negative DEF_ERR_* code and leaves a
+ *     human-readable message for def_last_error() (thread-local).  Nothing is
+ *     launched when validation fails.  No exception crosses this boundary.
+ *   - IEEE specials in the data propagate as the arithmetic above dictates; inputs are
+ *     not scanned.
+ */
+#ifndef DEF_B200_H
+#define DEF_B200_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct def_ctx def_ctx; /* opaque, owned by the library */
+
+enum { DEF_VARIANT_DEF = 0, DEF_VARIANT_DEF_A = 1, DEF_VARIANT_EF = 2 };
+
+enum {
+    DEF_OK = 0,
+    DEF_ERR_ARG = -1,         /* a size or hyper-parameter is out of range          */
+    DEF_ERR_NULL = -2,        /* a required pointer is NULL                         */
+    DEF_ERR_ALIGN = -3,       /* a pointer is not 4-byte aligned                    */
+    DEF_ERR_ALIAS = -4,       /* two tensors overlap                                */
+    DEF_ERR_DEVICE = -5,      /* no CUDA device, or not compute capability 10.x     */
+    DEF_ERR_CUDA = -6,        /* the CUDA runtime reported an error                 */
+    DEF_ERR_UNSUPPORTED = -7  /* a documented feature that is not implemented       */
+};
+
+#define DEF_MAX_WORKERS 64
+
+/*
+ * Algorithm 1's inputs.  d: model size; W: workers, 1..DEF_MAX_WORKERS; k: block
+ * length, 1 <= k <= d (compression ratio d/k); variant: DEF_VARIANT_*; lr: eta,
+ * finite; momentum: mu in [0, 1) (0 selects Algorithm 1 line 7 as printed);
+ * coeffs: NULL for the defaults {0.3, 0}, else coeffs[0] = lambda in [0, 1] (the
+ * detach coefficient; forced to 0 for DEF_VARIANT_EF) and coeffs[1] = weight decay,
+ * which must be 0 (the paper does not say where weight decay enters: fold it into
+ * the gradients; non-zero returns NULL with DEF_ERR_UNSUPPORTED).
+ * Returns NULL on failure (see def_last_error).  Touches no GPU: the device is
+ * checked by the first call that launches.
+ */
+def_ctx *def_create(int64_t d, int32_t W, int64_t k, int32_t variant, float lr, float momentum,
+                    const float *coeffs);
+
+/* Frees the handle and any device staging memory def_step_host allocated for it. */
+int def_destroy(def_ctx *ctx);
+
+/*
+ * One step (Algorithm 1 lines 7-10, Eq. 10), in place.
+ *   params [d]     x_t      -> x_{t+1}   (only the k block coordinates are touched)
+ *   grads  [W, d]  g_{k,t}     read only
+ *   errors [W, d]  e_{k,t}  -> e_{k,t+1}
+ *   mom    [W, d]  m_{k,t}  -> m_{k,t+1}; NULL if and only if momentum == 0
+ *   step, seed     t and the shared seed: the block start is a pure function of both
+ * The caller zeroes errors and mom before step 0 (Algorithm 1's initialisation).
+ * 16-byte aligned pointers with d % 4 == 0 run on 128-bit accesses; 8-byte / d % 2
+ * and 4-byte alignment are accepted and run on narrower accesses.
+ * Errors: DEF_ERR_NULL, DEF_ERR_ALIGN, DEF_ERR_ALIAS (any two of the four tensors
+ * overlap), DEF_ERR_DEVICE, DEF_ERR_CUDA (launch failure).
+ */
+int def_step(def_ctx *ctx, float *params, const float *grads, float *errors, float *mom,
+             uint64_t step, uint64_t seed);
+
+/*
+ * The same step on a contiguous range of coordinates [j0, j0 + n) of the
+ * d-dimensional problem: every operation of the step is separate per coordinate, so
+ * a model can be cut by columns across GPUs, or streamed through the GPU in pieces,
+ * with no exchange between the pieces.  params points at the n local coordinates;
+ * grads / errors / mom point at local [W, n] tensors with row stride ld >= n floats.
+ * The block start is still drawn over the whole d.  0 <= j0, j0 + n <= d.
+ */
+int def_step_columns(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, float *params,
+                     const float *grads, float *errors, float *mom, uint64_t step,
+                     uint64_t seed);
+
+/*
+ * One step with every tensor in HOST memory (pinned memory is much faster; pageable
+ * works).  The library streams column ranges through device staging buffers it owns
+ * (allocated on the first call, sized from the free device memory, freed by
+ * def_destroy): host->device copy, def_step_columns' kernel and device->host copy of
+ * successive ranges overlap on three streams.  Blocks until params_host,
+ * errors_host and mom_host hold the results.  Same shapes as def_step.
+ */
+int def_step_host(def_ctx *ctx, float *params_host, const float *grads_host, float *errors_host,
+                  float *mom_host, uint64_t step, uint64_t seed);
+
+/* def_step_columns with every tensor in host memory (same streaming as def_step_host):
+ * coordinates [j0, j0 + n) of the model, local [W, n] tensors with row stride ld. */
+int def_step_columns_host(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, float *params_host,
+                          const float *grads_host, float *errors_host, float *mom_host,
+                          uint64_t step, uint64_t seed);
+
+/* The stream device-pointer calls enqueue on (a cudaStream_t; NULL = legacy default). */
+int def_set_stream(def_ctx *ctx, void *cuda_stream);
+
+/* Learning-rate schedules: eta may change between steps. */
+int def_set_lr(def_ctx *ctx, float lr);
+
+/*
+ * The block start s_t in [0, d) that a step with (step, seed) uses, computed on the
+ * host by the library's own Philox4x32-10: key = (seed low, seed high), counter =
+ * (step low, step high, 0x52424753, 0), r = word0 | word1 << 32, s = floor(r d / 2^64).
+ */
+int def_block_start(const def_ctx *ctx, uint64_t step, uint64_t seed, int64_t *start_out);
+
+/*
+ * The same start computed by the device code the step kernels use, for a batch:
+ * starts_out[i] = start(seeds[i], steps[i], ds[i]).  All four are device arrays of
+ * n elements (uint64, uint64, int64, int64); ds[i] >= 1.  Enqueued on `cuda_stream`.
+ */
+int def_block_start_device(const uint64_t *seeds, const uint64_t *steps, const int64_t *ds,
+                           int64_t n, int64_t *starts_out, void *cuda_stream);
+
+/* Kernels this context has launched so far (every launch of every call). */
+int def_launch_count(const def_ctx *ctx, int64_t *count_out);
+
+/* Message of the last failure on this thread ("" if none). */
+const char *def_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DEF_B200_H */

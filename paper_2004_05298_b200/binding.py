@@ -1,0 +1,186 @@
+"""Thin ctypes binding of libdef_b200.so: the same entry points as include/def.h, taking
+torch tensors.  It checks dtype / contiguity / device / shape and passes data pointers;
+every step of the method runs inside the library's CUDA kernels.  There is no CPU or
+eager fallback: if the library cannot be built or loaded, importing fails loudly."""
+import ctypes
+import os
+
+import torch
+
+from . import build as _build
+
+DEF_VARIANT_DEF, DEF_VARIANT_DEF_A, DEF_VARIANT_EF = 0, 1, 2
+DEF_OK = 0
+DEF_ERR_ARG, DEF_ERR_NULL, DEF_ERR_ALIGN, DEF_ERR_ALIAS = -1, -2, -3, -4
+DEF_ERR_DEVICE, DEF_ERR_CUDA, DEF_ERR_UNSUPPORTED = -5, -6, -7
+DEF_MAX_WORKERS = 64
+
+_i64, _u64, _i32, _f32, _ptr = (ctypes.c_int64, ctypes.c_uint64, ctypes.c_int32, ctypes.c_float,
+                                ctypes.c_void_p)
+
+# name -> (restype, argtypes): every symbol include/def.h declares
+SIGNATURES = {
+    "def_create": (_ptr, [_i64, _i32, _i64, _i32, _f32, _f32, _ptr]),
+    "def_destroy": (ctypes.c_int, [_ptr]),
+    "def_step": (ctypes.c_int, [_ptr, _ptr, _ptr, _ptr, _ptr, _u64, _u64]),
+    "def_step_columns": (ctypes.c_int, [_ptr, _i64, _i64, _i64, _ptr, _ptr, _ptr, _ptr, _u64, _u64]),
+    "def_step_host": (ctypes.c_int, [_ptr, _ptr, _ptr, _ptr, _ptr, _u64, _u64]),
+    "def_step_columns_host": (ctypes.c_int, [_ptr, _i64, _i64, _i64, _ptr, _ptr, _ptr, _ptr, _u64, _u64]),
+    "def_set_stream": (ctypes.c_int, [_ptr, _ptr]),
+    "def_set_lr": (ctypes.c_int, [_ptr, _f32]),
+    "def_block_start": (ctypes.c_int, [_ptr, _u64, _u64, _ptr]),
+    "def_block_start_device": (ctypes.c_int, [_ptr, _ptr, _ptr, _i64, _ptr, _ptr]),
+    "def_launch_count": (ctypes.c_int, [_ptr, _ptr]),
+    "def_last_error": (ctypes.c_char_p, []),
+}
+
+
+class DefError(RuntimeError):
+    def __init__(self, code, message):
+        super().__init__("def error %d: %s" % (code, message))
+        self.code = code
+
+
+def _load():
+    path = _build.build()
+    if not os.path.exists(path):
+        raise ImportError("libdef_b200.so is missing and could not be built")
+    lib = ctypes.CDLL(path)
+    for name, (restype, argtypes) in SIGNATURES.items():
+        fn = getattr(lib, name)          # AttributeError if the library lacks a declared symbol
+        fn.restype = restype
+        fn.argtypes = argtypes
+    return lib
+
+
+lib = _load()
+LIB_PATH = _build.LIB
+
+
+def def_last_error():
+    return lib.def_last_error().decode()
+
+
+def _check(rc):
+    if rc != DEF_OK:
+        raise DefError(rc, def_last_error())
+
+
+def _dev(t, name, shape=None, dtype=torch.float32, optional=False):
+    if t is None:
+        if optional:
+            return None
+        raise DefError(DEF_ERR_NULL, "%s is None" % name)
+    if not isinstance(t, torch.Tensor) or t.dtype != dtype or not t.is_contiguous():
+        raise TypeError("%s must be a contiguous %s torch tensor" % (name, dtype))
+    if not t.is_cuda:
+        raise TypeError("%s must live on the GPU" % name)
+    if shape is not None and tuple(t.shape) != tuple(shape):
+        raise ValueError("%s has shape %s, expected %s" % (name, tuple(t.shape), tuple(shape)))
+    return t.data_ptr()
+
+
+def _host(t, name, shape, optional=False):
+    if t is None:
+        if optional:
+            return None
+        raise DefError(DEF_ERR_NULL, "%s is None" % name)
+    if not isinstance(t, torch.Tensor) or t.dtype != torch.float32 or not t.is_contiguous() or t.is_cuda:
+        raise TypeError("%s must be a contiguous float32 CPU tensor" % name)
+    if tuple(t.shape) != tuple(shape):
+        raise ValueError("%s has shape %s, expected %s" % (name, tuple(t.shape), tuple(shape)))
+    return t.data_ptr()
+
+
+class DefCtx:
+    """Owner of one def_ctx handle (freed by def_destroy or when collected)."""
+
+    def __init__(self, handle, d, W, k, variant, lr, momentum):
+        self.handle = handle
+        self.d, self.W, self.k, self.variant, self.lr, self.momentum = d, W, k, variant, lr, momentum
+
+    def __del__(self):
+        if getattr(self, "handle", None):
+            lib.def_destroy(self.handle)
+            self.handle = None
+
+
+def def_create(d, W, k, variant, lr, momentum, coeffs=None):
+    arr = None
+    if coeffs is not None:
+        arr = (ctypes.c_float * 2)(float(coeffs[0]), float(coeffs[1]))
+    handle = lib.def_create(int(d), int(W), int(k), int(variant), float(lr), float(momentum), arr)
+    if not handle:
+        msg = def_last_error()
+        raise DefError(DEF_ERR_UNSUPPORTED if "weight decay" in msg else DEF_ERR_ARG, msg)
+    return DefCtx(handle, int(d), int(W), int(k), int(variant), float(lr), float(momentum))
+
+
+def def_destroy(ctx):
+    if ctx.handle:
+        rc = lib.def_destroy(ctx.handle)
+        ctx.handle = None
+        _check(rc)
+
+
+def def_set_stream(ctx, stream):
+    """stream: a torch.cuda.Stream, a raw cudaStream_t integer, or None (legacy default)."""
+    raw = stream.cuda_stream if isinstance(stream, torch.cuda.Stream) else (stream or 0)
+    _check(lib.def_set_stream(ctx.handle, ctypes.c_void_p(raw)))
+
+
+def def_set_lr(ctx, lr):
+    _check(lib.def_set_lr(ctx.handle, float(lr)))
+    ctx.lr = float(lr)
+
+
+def def_step(ctx, params, grads, errors, mom, step, seed):
+    d, W = ctx.d, ctx.W
+    _check(lib.def_step(ctx.handle, _dev(params, "params", (d,)), _dev(grads, "grads", (W, d)),
+                        _dev(errors, "errors", (W, d)), _dev(mom, "mom", (W, d), optional=True),
+                        int(step), int(seed)))
+
+
+def def_step_columns(ctx, j0, n, ld, params, grads, errors, mom, step, seed):
+    """params: [n]; grads / errors / mom: [W, ld] (a rank's local column shard)."""
+    W = ctx.W
+    _check(lib.def_step_columns(ctx.handle, int(j0), int(n), int(ld), _dev(params, "params", (n,)),
+                                _dev(grads, "grads", (W, ld)), _dev(errors, "errors", (W, ld)),
+                                _dev(mom, "mom", (W, ld), optional=True), int(step), int(seed)))
+
+
+def def_step_host(ctx, params, grads, errors, mom, step, seed):
+    d, W = ctx.d, ctx.W
+    _check(lib.def_step_host(ctx.handle, _host(params, "params", (d,)), _host(grads, "grads", (W, d)),
+                             _host(errors, "errors", (W, d)), _host(mom, "mom", (W, d), optional=True),
+                             int(step), int(seed)))
+
+
+def def_step_columns_host(ctx, j0, n, ld, params, grads, errors, mom, step, seed):
+    W = ctx.W
+    _check(lib.def_step_columns_host(ctx.handle, int(j0), int(n), int(ld), _host(params, "params", (n,)),
+                                     _host(grads, "grads", (W, ld)), _host(errors, "errors", (W, ld)),
+                                     _host(mom, "mom", (W, ld), optional=True), int(step), int(seed)))
+
+
+def def_block_start(ctx, step, seed):
+    out = ctypes.c_int64(-1)
+    _check(lib.def_block_start(ctx.handle, int(step), int(seed), ctypes.byref(out)))
+    return int(out.value)
+
+
+def def_block_start_device(seeds, steps, ds, starts_out, stream=None):
+    """seeds, steps: uint64 bit patterns held in int64 CUDA tensors; ds, starts_out: int64."""
+    n = seeds.numel()
+    raw = stream.cuda_stream if isinstance(stream, torch.cuda.Stream) else (stream or 0)
+    _check(lib.def_block_start_device(_dev(seeds, "seeds", (n,), torch.int64),
+                                      _dev(steps, "steps", (n,), torch.int64),
+                                      _dev(ds, "ds", (n,), torch.int64), n,
+                                      _dev(starts_out, "starts_out", (n,), torch.int64),
+                                      ctypes.c_void_p(raw)))
+
+
+def def_launch_count(ctx):
+    out = ctypes.c_int64(0)
+    _check(lib.def_launch_count(ctx.handle, ctypes.byref(out)))
+    return int(out.value)

@@ -1,0 +1,401 @@
+// C boundary of the DEF / DEF-A / EF step library (see include/def.h): argument
+// validation, kernel selection and launch, and the host-memory streaming path.
+#include "../../include/def.h"
+#include "def_kernels.cuh"
+
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+namespace {
+
+thread_local char g_last_error[512] = "";
+
+int fail(int code, const char *fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_last_error, sizeof(g_last_error), fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+int cuda_fail(cudaError_t err, const char *what) {
+    return fail(DEF_ERR_CUDA, "%s: %s", what, cudaGetErrorString(err));
+}
+
+constexpr int kThreads = 256;
+constexpr int kHostSlots = 3;  // staging slots of the host-memory path
+
+struct HostSlot {
+    float *x = nullptr, *g = nullptr, *e = nullptr, *m = nullptr;
+    cudaEvent_t loaded = nullptr, computed = nullptr, drained = nullptr;
+    bool used = false;
+};
+
+}  // namespace
+
+struct def_ctx {
+    int64_t d = 0, k = 0;
+    int32_t W = 0, variant = 0;
+    float lr = 0.f, momentum = 0.f, lambda = 0.3f;
+    cudaStream_t stream = nullptr;
+    int64_t launches = 0;
+    // device facts, filled by the first launching call
+    bool device_checked = false;
+    int device = -1;
+    int sm_count = 0;
+    // host-memory path
+    bool host_ready = false;
+    int64_t host_chunk = 0;  // coordinates per staging slot (multiple of 4)
+    HostSlot slots[kHostSlots];
+    cudaStream_t s_h2d = nullptr, s_run = nullptr, s_d2h = nullptr;
+};
+
+namespace {
+
+int check_device(def_ctx *ctx) {
+    int dev = -1;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) {
+        cudaGetLastError();
+        return fail(DEF_ERR_DEVICE, "no usable CUDA device: %s", cudaGetErrorString(err));
+    }
+    if (ctx->device_checked && ctx->device == dev) return DEF_OK;
+    cudaDeviceProp prop;
+    err = cudaGetDeviceProperties(&prop, dev);
+    if (err != cudaSuccess) {
+        cudaGetLastError();
+        return fail(DEF_ERR_DEVICE, "cannot query device %d: %s", dev, cudaGetErrorString(err));
+    }
+    if (prop.major != 10)
+        return fail(DEF_ERR_DEVICE, "device %d is compute capability %d.%d; this library is built for 10.x (sm_100a)",
+                    dev, prop.major, prop.minor);
+    ctx->device = dev;
+    ctx->sm_count = prop.multiProcessorCount;
+    ctx->device_checked = true;
+    return DEF_OK;
+}
+
+bool overlaps(const void *a, size_t a_bytes, const void *b, size_t b_bytes) {
+    const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
+    return a0 < b0 + b_bytes && b0 < a0 + a_bytes;
+}
+
+// Bytes spanned by a [W, n] view with row stride ld, and by x[n].
+size_t span_rows(int64_t W, int64_t n, int64_t ld) {
+    return ((size_t)(W - 1) * (size_t)ld + (size_t)n) * sizeof(float);
+}
+
+int validate_tensors(const def_ctx *ctx, int64_t n, int64_t ld, const float *x, const float *g,
+                     const float *e, const float *m) {
+    if (!x || !g || !e) return fail(DEF_ERR_NULL, "params, grads and errors must not be NULL");
+    if (ctx->momentum != 0.f && !m)
+        return fail(DEF_ERR_NULL, "mom must not be NULL when momentum != 0");
+    if (ctx->momentum == 0.f && m)
+        return fail(DEF_ERR_ARG, "mom must be NULL when momentum == 0");
+    const void *ptrs[4] = {x, g, e, m};
+    const char *names[4] = {"params", "grads", "errors", "mom"};
+    for (int i = 0; i < 4; ++i)
+        if (ptrs[i] && ((uintptr_t)ptrs[i] & 3u))
+            return fail(DEF_ERR_ALIGN, "%s is not 4-byte aligned", names[i]);
+    const size_t bytes[4] = {(size_t)n * sizeof(float), span_rows(ctx->W, n, ld),
+                             span_rows(ctx->W, n, ld), span_rows(ctx->W, n, ld)};
+    for (int i = 0; i < 4; ++i)
+        for (int j = i + 1; j < 4; ++j)
+            if (ptrs[i] && ptrs[j] && overlaps(ptrs[i], bytes[i], ptrs[j], bytes[j]))
+                return fail(DEF_ERR_ALIAS, "%s and %s overlap", names[i], names[j]);
+    return DEF_OK;
+}
+
+// Widest access every row of the view supports.
+int vector_width(int64_t ld, const float *x, const float *g, const float *e, const float *m) {
+    uintptr_t bits = (uintptr_t)x | (uintptr_t)g | (uintptr_t)e | (uintptr_t)m;
+    if ((bits & 15u) == 0 && ld % 4 == 0) return 4;
+    if ((bits & 7u) == 0 && ld % 2 == 0) return 2;
+    return 1;
+}
+
+template <int V, bool MOM>
+cudaError_t launch_one(const def_ctx *ctx, const defk::StepArgs &a, cudaStream_t stream) {
+    // 4 rows in flight per thread: 12 independent 16-byte loads before the first use.
+    constexpr int U = 4;
+    const int64_t groups = a.n / V;
+    if (groups == 0) return cudaSuccess;
+    const int64_t want = (groups + kThreads - 1) / kThreads;
+    // a few waves of whole-SM multiples; beyond that the grid-stride loop takes over
+    const int64_t cap = (int64_t)ctx->sm_count * 8 * 4;
+    const unsigned grid = (unsigned)(want < cap ? want : cap);
+    defk::def_step_kernel<V, MOM, U><<<grid, kThreads, 0, stream>>>(a);
+    return cudaGetLastError();
+}
+
+template <int V>
+cudaError_t launch_v(const def_ctx *ctx, const defk::StepArgs &a, cudaStream_t stream) {
+    return a.m ? launch_one<V, true>(ctx, a, stream) : launch_one<V, false>(ctx, a, stream);
+}
+
+// Enqueue the step on local coordinates [0, n) of a view; counts launches.
+int enqueue_columns(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, float *x, const float *g,
+                    float *e, float *m, uint64_t step, uint64_t seed, cudaStream_t stream) {
+    if (n == 0) return DEF_OK;
+    defk::StepArgs a;
+    a.x = x; a.g = g; a.e = e; a.m = m;
+    a.n = n; a.ld = ld; a.d = ctx->d; a.j0 = j0; a.k = ctx->k; a.W = ctx->W;
+    a.eta = ctx->lr; a.mu = ctx->momentum; a.W_float = (float)ctx->W;
+    a.seed = seed; a.step = step;
+    const int V = vector_width(ld, x, g, e, m);
+    cudaError_t err = cudaSuccess;
+    const int64_t body = n - n % V;
+    if (body > 0) {
+        a.n = body;
+        err = V == 4 ? launch_v<4>(ctx, a, stream) : V == 2 ? launch_v<2>(ctx, a, stream)
+                                                              : launch_v<1>(ctx, a, stream);
+        if (err != cudaSuccess) return cuda_fail(err, "def_step kernel launch");
+        ctx->launches += 1;
+    }
+    if (body < n) {  // the last n % V coordinates, one float at a time
+        defk::StepArgs t = a;
+        t.x = x + body; t.g = g + body; t.e = e + body; t.m = m ? m + body : nullptr;
+        t.n = n - body; t.j0 = j0 + body;
+        err = launch_v<1>(ctx, t, stream);
+        if (err != cudaSuccess) return cuda_fail(err, "def_step tail kernel launch");
+        ctx->launches += 1;
+    }
+    return DEF_OK;
+}
+
+void free_host_path(def_ctx *ctx) {
+    for (HostSlot &s : ctx->slots) {
+        if (s.x) cudaFree(s.x);
+        if (s.g) cudaFree(s.g);
+        if (s.e) cudaFree(s.e);
+        if (s.m) cudaFree(s.m);
+        if (s.loaded) cudaEventDestroy(s.loaded);
+        if (s.computed) cudaEventDestroy(s.computed);
+        if (s.drained) cudaEventDestroy(s.drained);
+        s = HostSlot();
+    }
+    if (ctx->s_h2d) cudaStreamDestroy(ctx->s_h2d);
+    if (ctx->s_run) cudaStreamDestroy(ctx->s_run);
+    if (ctx->s_d2h) cudaStreamDestroy(ctx->s_d2h);
+    ctx->s_h2d = ctx->s_run = ctx->s_d2h = nullptr;
+    ctx->host_ready = false;
+}
+
+int prepare_host_path(def_ctx *ctx) {
+    if (ctx->host_ready) return DEF_OK;
+    size_t free_b = 0, total_b = 0;
+    cudaError_t err = cudaMemGetInfo(&free_b, &total_b);
+    if (err != cudaSuccess) return cuda_fail(err, "cudaMemGetInfo");
+    // one slot holds x plus g, e (and m) for `chunk` coordinates; aim at 128 MiB of
+    // row data per slot, but never more than a quarter of the free memory in total
+    const int rows = ctx->W * (ctx->momentum != 0.f ? 3 : 2) + 1;
+    int64_t chunk = (int64_t)((128u << 20) / (sizeof(float) * (size_t)rows));
+    const int64_t by_memory = (int64_t)(free_b / 4 / kHostSlots / (sizeof(float) * (size_t)rows));
+    if (chunk > by_memory) chunk = by_memory;
+    if (chunk > ctx->d) chunk = ctx->d;
+    chunk = (chunk + 3) / 4 * 4;
+    if (chunk < 4) return fail(DEF_ERR_CUDA, "not enough free device memory for staging buffers");
+    const size_t row_bytes = (size_t)chunk * sizeof(float);
+    for (HostSlot &s : ctx->slots) {
+        if ((err = cudaMalloc(&s.x, row_bytes)) != cudaSuccess ||
+            (err = cudaMalloc(&s.g, row_bytes * ctx->W)) != cudaSuccess ||
+            (err = cudaMalloc(&s.e, row_bytes * ctx->W)) != cudaSuccess ||
+            (ctx->momentum != 0.f && (err = cudaMalloc(&s.m, row_bytes * ctx->W)) != cudaSuccess) ||
+            (err = cudaEventCreateWithFlags(&s.loaded, cudaEventDisableTiming)) != cudaSuccess ||
+            (err = cudaEventCreateWithFlags(&s.computed, cudaEventDisableTiming)) != cudaSuccess ||
+            (err = cudaEventCreateWithFlags(&s.drained, cudaEventDisableTiming)) != cudaSuccess) {
+            free_host_path(ctx);
+            return cuda_fail(err, "allocating staging buffers");
+        }
+    }
+    if ((err = cudaStreamCreateWithFlags(&ctx->s_h2d, cudaStreamNonBlocking)) != cudaSuccess ||
+        (err = cudaStreamCreateWithFlags(&ctx->s_run, cudaStreamNonBlocking)) != cudaSuccess ||
+        (err = cudaStreamCreateWithFlags(&ctx->s_d2h, cudaStreamNonBlocking)) != cudaSuccess) {
+        free_host_path(ctx);
+        return cuda_fail(err, "creating streams");
+    }
+    ctx->host_chunk = chunk;
+    ctx->host_ready = true;
+    return DEF_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *def_last_error(void) { return g_last_error; }
+
+def_ctx *def_create(int64_t d, int32_t W, int64_t k, int32_t variant, float lr, float momentum,
+                    const float *coeffs) {
+    g_last_error[0] = 0;
+    if (d < 1) { fail(DEF_ERR_ARG, "d must be >= 1 (got %lld)", (long long)d); return nullptr; }
+    if (W < 1 || W > DEF_MAX_WORKERS) {
+        fail(DEF_ERR_ARG, "W must be in 1..%d (got %d)", DEF_MAX_WORKERS, W);
+        return nullptr;
+    }
+    if (k < 1 || k > d) {
+        fail(DEF_ERR_ARG, "k must be in 1..d (got k=%lld, d=%lld)", (long long)k, (long long)d);
+        return nullptr;
+    }
+    if (variant != DEF_VARIANT_DEF && variant != DEF_VARIANT_DEF_A && variant != DEF_VARIANT_EF) {
+        fail(DEF_ERR_ARG, "unknown variant %d", variant);
+        return nullptr;
+    }
+    if (!std::isfinite(lr)) { fail(DEF_ERR_ARG, "lr must be finite"); return nullptr; }
+    if (!(momentum >= 0.f && momentum < 1.f)) {
+        fail(DEF_ERR_ARG, "momentum must be in [0, 1)");
+        return nullptr;
+    }
+    float lambda = 0.3f;
+    if (coeffs) {
+        lambda = coeffs[0];
+        if (!(lambda >= 0.f && lambda <= 1.f)) {
+            fail(DEF_ERR_ARG, "coeffs[0] (lambda) must be in [0, 1]");
+            return nullptr;
+        }
+        if (coeffs[1] != 0.f) {
+            fail(DEF_ERR_UNSUPPORTED, "coeffs[1] (weight decay) must be 0: fold weight decay into the gradients");
+            return nullptr;
+        }
+    }
+    if (variant == DEF_VARIANT_EF) lambda = 0.f;
+    def_ctx *ctx = new (std::nothrow) def_ctx();
+    if (!ctx) { fail(DEF_ERR_ARG, "out of host memory"); return nullptr; }
+    ctx->d = d; ctx->W = W; ctx->k = k; ctx->variant = variant;
+    ctx->lr = lr; ctx->momentum = momentum; ctx->lambda = lambda;
+    return ctx;
+}
+
+int def_destroy(def_ctx *ctx) {
+    if (!ctx) return fail(DEF_ERR_NULL, "ctx is NULL");
+    free_host_path(ctx);
+    delete ctx;
+    return DEF_OK;
+}
+
+int def_set_stream(def_ctx *ctx, void *cuda_stream) {
+    if (!ctx) return fail(DEF_ERR_NULL, "ctx is NULL");
+    ctx->stream = (cudaStream_t)cuda_stream;
+    return DEF_OK;
+}
+
+int def_set_lr(def_ctx *ctx, float lr) {
+    if (!ctx) return fail(DEF_ERR_NULL, "ctx is NULL");
+    if (!std::isfinite(lr)) return fail(DEF_ERR_ARG, "lr must be finite");
+    ctx->lr = lr;
+    return DEF_OK;
+}
+
+int def_block_start(const def_ctx *ctx, uint64_t step, uint64_t seed, int64_t *start_out) {
+    if (!ctx || !start_out) return fail(DEF_ERR_NULL, "ctx and start_out must not be NULL");
+    *start_out = defk::block_start(seed, step, ctx->d);
+    return DEF_OK;
+}
+
+int def_block_start_device(const uint64_t *seeds, const uint64_t *steps, const int64_t *ds,
+                           int64_t n, int64_t *starts_out, void *cuda_stream) {
+    if (!seeds || !steps || !ds || !starts_out) return fail(DEF_ERR_NULL, "NULL array");
+    if (n < 0) return fail(DEF_ERR_ARG, "n must be >= 0");
+    if (n == 0) return DEF_OK;
+    const int64_t blocks = (n + 255) / 256;
+    if (blocks > 0x7fffffffLL) return fail(DEF_ERR_ARG, "n too large");
+    defk::block_start_batch_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)cuda_stream>>>(
+        seeds, steps, ds, n, starts_out);
+    cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) return cuda_fail(err, "block start kernel launch");
+    return DEF_OK;
+}
+
+int def_launch_count(const def_ctx *ctx, int64_t *count_out) {
+    if (!ctx || !count_out) return fail(DEF_ERR_NULL, "ctx and count_out must not be NULL");
+    *count_out = ctx->launches;
+    return DEF_OK;
+}
+
+int def_step_columns(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, float *params,
+                     const float *grads, float *errors, float *mom, uint64_t step,
+                     uint64_t seed) {
+    if (!ctx) return fail(DEF_ERR_NULL, "ctx is NULL");
+    if (j0 < 0 || n < 0 || j0 > ctx->d || n > ctx->d - j0)
+        return fail(DEF_ERR_ARG, "column range [%lld, %lld) is outside [0, %lld)", (long long)j0,
+                    (long long)(j0 + n), (long long)ctx->d);
+    if (ld < n) return fail(DEF_ERR_ARG, "row stride ld=%lld is smaller than n=%lld", (long long)ld, (long long)n);
+    int rc = validate_tensors(ctx, n, ld, params, grads, errors, mom);
+    if (rc != DEF_OK) return rc;
+    if ((rc = check_device(ctx)) != DEF_OK) return rc;
+    return enqueue_columns(ctx, j0, n, ld, params, grads, errors, mom, step, seed, ctx->stream);
+}
+
+int def_step(def_ctx *ctx, float *params, const float *grads, float *errors, float *mom,
+             uint64_t step, uint64_t seed) {
+    if (!ctx) return fail(DEF_ERR_NULL, "ctx is NULL");
+    return def_step_columns(ctx, 0, ctx->d, ctx->d, params, grads, errors, mom, step, seed);
+}
+
+int def_step_host(def_ctx *ctx, float *params_host, const float *grads_host, float *errors_host,
+                  float *mom_host, uint64_t step, uint64_t seed) {
+    if (!ctx) return fail(DEF_ERR_NULL, "ctx is NULL");
+    return def_step_columns_host(ctx, 0, ctx->d, ctx->d, params_host, grads_host, errors_host,
+                                 mom_host, step, seed);
+}
+
+int def_step_columns_host(def_ctx *ctx, int64_t c0, int64_t cols, int64_t ld, float *params_host,
+                          const float *grads_host, float *errors_host, float *mom_host,
+                          uint64_t step, uint64_t seed) {
+    if (!ctx) return fail(DEF_ERR_NULL, "ctx is NULL");
+    if (c0 < 0 || cols < 0 || c0 > ctx->d || cols > ctx->d - c0)
+        return fail(DEF_ERR_ARG, "column range [%lld, %lld) is outside [0, %lld)", (long long)c0,
+                    (long long)(c0 + cols), (long long)ctx->d);
+    if (ld < cols) return fail(DEF_ERR_ARG, "row stride ld=%lld is smaller than n=%lld", (long long)ld, (long long)cols);
+    int rc = validate_tensors(ctx, cols, ld, params_host, grads_host, errors_host, mom_host);
+    if (rc != DEF_OK) return rc;
+    if ((rc = check_device(ctx)) != DEF_OK) return rc;
+    if ((rc = prepare_host_path(ctx)) != DEF_OK) return rc;
+
+    const int64_t d = cols, chunk = ctx->host_chunk;   // local coordinates 0..cols-1
+    const int W = ctx->W;
+    const size_t host_pitch = (size_t)ld * sizeof(float);
+    const size_t dev_pitch = (size_t)chunk * sizeof(float);
+    cudaError_t err = cudaSuccess;
+    int64_t piece = 0;
+    for (int64_t j0 = 0; j0 < d; j0 += chunk, ++piece) {
+        HostSlot &s = ctx->slots[piece % kHostSlots];
+        const int64_t n = (d - j0 < chunk) ? d - j0 : chunk;
+        const size_t width = (size_t)n * sizeof(float);
+        // the slot's previous piece must have left the device before it is overwritten
+        if (s.used && (err = cudaStreamWaitEvent(ctx->s_h2d, s.drained, 0)) != cudaSuccess) break;
+        if ((err = cudaMemcpyAsync(s.x, params_host + j0, width, cudaMemcpyHostToDevice, ctx->s_h2d)) != cudaSuccess) break;
+        if ((err = cudaMemcpy2DAsync(s.g, dev_pitch, grads_host + j0, host_pitch, width, W, cudaMemcpyHostToDevice, ctx->s_h2d)) != cudaSuccess) break;
+        if ((err = cudaMemcpy2DAsync(s.e, dev_pitch, errors_host + j0, host_pitch, width, W, cudaMemcpyHostToDevice, ctx->s_h2d)) != cudaSuccess) break;
+        if (mom_host && (err = cudaMemcpy2DAsync(s.m, dev_pitch, mom_host + j0, host_pitch, width, W, cudaMemcpyHostToDevice, ctx->s_h2d)) != cudaSuccess) break;
+        if ((err = cudaEventRecord(s.loaded, ctx->s_h2d)) != cudaSuccess) break;
+
+        if ((err = cudaStreamWaitEvent(ctx->s_run, s.loaded, 0)) != cudaSuccess) break;
+        rc = enqueue_columns(ctx, c0 + j0, n, chunk, s.x, s.g, s.e, mom_host ? s.m : nullptr, step, seed, ctx->s_run);
+        if (rc != DEF_OK) break;
+        if ((err = cudaEventRecord(s.computed, ctx->s_run)) != cudaSuccess) break;
+
+        if ((err = cudaStreamWaitEvent(ctx->s_d2h, s.computed, 0)) != cudaSuccess) break;
+        if ((err = cudaMemcpyAsync(params_host + j0, s.x, width, cudaMemcpyDeviceToHost, ctx->s_d2h)) != cudaSuccess) break;
+        if ((err = cudaMemcpy2DAsync(errors_host + j0, host_pitch, s.e, dev_pitch, width, W, cudaMemcpyDeviceToHost, ctx->s_d2h)) != cudaSuccess) break;
+        if (mom_host && (err = cudaMemcpy2DAsync(mom_host + j0, host_pitch, s.m, dev_pitch, width, W, cudaMemcpyDeviceToHost, ctx->s_d2h)) != cudaSuccess) break;
+        if ((err = cudaEventRecord(s.drained, ctx->s_d2h)) != cudaSuccess) break;
+        s.used = true;
+    }
+    // drain everything that was enqueued, also after a failure
+    cudaError_t e1 = cudaStreamSynchronize(ctx->s_h2d);
+    cudaError_t e2 = cudaStreamSynchronize(ctx->s_run);
+    cudaError_t e3 = cudaStreamSynchronize(ctx->s_d2h);
+    if (rc != DEF_OK) return rc;
+    if (err != cudaSuccess) return cuda_fail(err, "def_step_host");
+    if (e1 != cudaSuccess) return cuda_fail(e1, "def_step_host (host->device stream)");
+    if (e2 != cudaSuccess) return cuda_fail(e2, "def_step_host (compute stream)");
+    if (e3 != cudaSuccess) return cuda_fail(e3, "def_step_host (device->host stream)");
+    return DEF_OK;
+}
+
+}  // extern "C"

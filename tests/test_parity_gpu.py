@@ -1,0 +1,403 @@
+"""GPU parity: the CUDA library, called through its C boundary, against the CPU oracle
+on the same seeded inputs.
+
+Bars: block starts and masks bit-exact; params, errors and momentum within a maximum
+relative error of 1e-5 of the fp32 oracle (zeros must be zeros) after the workload's
+steps -- the library performs the same roundings in the same order as the oracle, so
+the difference is expected to be exactly 0 and the tests also report whether it is --
+and within 1e-5 of the tensor's scale of the fp64 shadow.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2004_05298_b200 import workloads as WL
+
+pytestmark = pytest.mark.gpu
+
+REL_TOL = 1e-5          # maximum element-wise relative error vs the fp32 oracle
+SHADOW_TOL = 1e-5       # maximum error vs the fp64 shadow, relative to the tensor's scale
+
+
+@pytest.fixture(scope="module")
+def B():
+    if not torch.cuda.is_available():
+        pytest.fail("these tests need a CUDA device (run with -m 'not gpu' on a CPU box)")
+    from paper_2004_05298_b200 import binding
+    return binding
+
+
+def compare(a, b, what, rel_tol=REL_TOL):
+    """a: library result, b: fp32 oracle result (numpy float32 arrays of one shape)."""
+    a = np.asarray(a); b = np.asarray(b)
+    assert a.shape == b.shape, what
+    both_nan = np.isnan(a) & np.isnan(b)
+    a = np.where(both_nan, 0, a); b = np.where(both_nan, 0, b)
+    assert np.array_equal(a == 0, b == 0), "%s: zero pattern differs" % what
+    nz = b != 0
+    if nz.any():
+        with np.errstate(invalid="ignore", over="ignore"):
+            rel = np.abs(a[nz].astype(np.float64) - b[nz].astype(np.float64)) / np.abs(b[nz].astype(np.float64))
+        rel = np.where(a[nz] == b[nz], 0.0, rel)       # equal infinities
+        m1 = float(np.max(rel))
+        assert m1 <= rel_tol, "%s: max relative error %.3e > %.1e" % (what, m1, rel_tol)
+    return bool(np.array_equal(a, b))
+
+
+def compare_shadow(a, b64, what, tol=SHADOW_TOL):
+    scale = float(np.max(np.abs(b64)))
+    if scale == 0.0:
+        assert not np.any(a), what
+        return
+    err = float(np.max(np.abs(a.astype(np.float64) - b64)))
+    assert err <= tol * scale, "%s: %.3e of scale vs the fp64 shadow" % (what, err / scale)
+
+
+def guarded(shape, device, fill=-12345.0, guard=64, offset=0):
+    """A tensor of `shape` inside a larger sentinel-filled buffer; `offset` floats shift its
+    start off the buffer's 16-byte grid.  Returns (view, check) where check() asserts that
+    nothing outside the view was written."""
+    n = int(np.prod(shape))
+    buf = torch.full((n + 2 * guard + 8,), fill, dtype=torch.float32, device=device)
+    start = guard + offset
+    view = buf[start:start + n].view(*shape)
+
+    def check():
+        assert bool((buf[:start] == fill).all()) and bool((buf[start + n:] == fill).all()), \
+            "a write landed outside the tensor"
+    return view, check
+
+
+def find_steps(d, k, seed, want):
+    """Steps whose block start satisfies want(s), by scanning the oracle's sampler."""
+    out = []
+    t = 0
+    while len(out) < 2 and t < 200000:
+        if want(oracle.block_start(seed, t, d)):
+            out.append(t)
+        t += 1
+    return out
+
+
+# ---------------------------------------------------------------------------
+# a1: the sampler, bit for bit
+# ---------------------------------------------------------------------------
+def test_block_start_device_matches_oracle(B):
+    n = 1 << 20
+    rng = np.random.default_rng(2024)
+    seeds = rng.integers(0, 2 ** 64, size=n, dtype=np.uint64)
+    steps = rng.integers(0, 2 ** 64, size=n, dtype=np.uint64)
+    seeds[: n // 2] %= 8                      # the small seeds and steps real runs use
+    steps[: n // 2] %= 100000
+    choices = np.array([1, 2, 3, 855770, 1000000, 11689512, 25557032, 138357544, 2 ** 40 + 7, 2 ** 62],
+                       dtype=np.int64)
+    ds = choices[rng.integers(0, len(choices), size=n)]
+    dev = torch.device("cuda")
+    out = torch.empty(n, dtype=torch.int64, device=dev)
+    B.def_block_start_device(torch.from_numpy(seeds.view(np.int64)).to(dev),
+                             torch.from_numpy(steps.view(np.int64)).to(dev),
+                             torch.from_numpy(ds).to(dev), out)
+    got = out.cpu().numpy()
+    f = oracle.default().lib.def_oracle_block_start
+    want = np.fromiter((f(int(a), int(b), int(c)) for a, b, c in zip(seeds, steps, ds)), dtype=np.int64, count=n)
+    assert np.array_equal(got, want)
+
+
+# ---------------------------------------------------------------------------
+# whole-tensor parity on shapes chosen to hit every code path
+# ---------------------------------------------------------------------------
+def run_whole(B, d, W, k, steps, momentum, seed, lr=0.1, offsets=(0, 0, 0, 0), sigma=0.1,
+              variant=0, special=None):
+    dev = torch.device("cuda")
+    rng = np.random.default_rng(d * 31 + W * 7 + k)
+    x, cx = guarded((d,), dev, offset=offsets[0])
+    g, cg = guarded((W, d), dev, offset=offsets[1])
+    e, ce = guarded((W, d), dev, offset=offsets[2])
+    x.copy_(torch.from_numpy((0.05 * rng.standard_normal(d)).astype(np.float32)))
+    e.zero_()
+    m = cm = None
+    if momentum:
+        m, cm = guarded((W, d), dev, offset=offsets[3])
+        m.zero_()
+    xo = x.cpu().numpy().copy(); eo = np.zeros((W, d), np.float32)
+    mo = np.zeros((W, d), np.float32) if momentum else None
+    x64 = xo.astype(np.float64); e64 = eo.astype(np.float64)
+    m64 = mo.astype(np.float64) if momentum else None
+    ctx = B.def_create(d, W, k, variant, lr, momentum)
+    exact = True
+    for t in steps:
+        gh = (sigma * rng.standard_normal((W, d))).astype(np.float32)
+        if special is not None:
+            special(gh, t)
+        g.copy_(torch.from_numpy(gh))
+        B.def_step(ctx, x, g, e, m, t, seed)
+        s = oracle.block_start(seed, t, d)
+        assert B.def_block_start(ctx, t, seed) == s
+        oracle.step(xo, gh, eo, mo, d=d, k=k, s=s, eta=lr, mu=momentum)
+        oracle.step(x64, gh.astype(np.float64), e64, m64, d=d, k=k, s=s, eta=lr, mu=momentum)
+        # the mask, bit-exact: after a step e' is +0 exactly on the block
+        mask = oracle.block_mask(d, k, s)
+        eg = e.cpu().numpy()
+        if special is None:
+            assert np.array_equal(eg == 0, np.broadcast_to(mask, (W, d))), "block mask differs at step %d" % t
+        assert np.array_equal(g.cpu().numpy(), gh, equal_nan=True), "grads must not be written"
+    torch.cuda.synchronize()
+    for chk in (cx, cg, ce, cm):
+        if chk:
+            chk()
+    exact &= compare(x.cpu().numpy(), xo, "params")
+    exact &= compare(e.cpu().numpy(), eo, "errors")
+    if momentum:
+        exact &= compare(m.cpu().numpy(), mo, "mom")
+    if special is None:
+        compare_shadow(x.cpu().numpy(), x64, "params")
+        compare_shadow(e.cpu().numpy(), e64, "errors")
+        if momentum:
+            compare_shadow(m.cpu().numpy(), m64, "mom")
+    B.def_destroy(ctx)
+    return exact
+
+
+SHAPES = [
+    # d, W, k
+    (1, 1, 1), (2, 3, 1), (5, 3, 2), (8, 2, 3), (1023, 3, 1), (1024, 4, 1024), (1025, 5, 1024),
+    (4099, 7, 100), (4100, 16, 4099), (100003, 9, 3125), (65536, 64, 777), (300000, 13, 150000),
+]
+
+
+@pytest.mark.parametrize("d,W,k", SHAPES)
+@pytest.mark.parametrize("momentum", [0.9, 0.0])
+def test_small_shapes(B, d, W, k, momentum):
+    seed = 11
+    wrap = find_steps(d, k, seed, lambda s: s + k > d)          # block wraps past the end
+    tail = find_steps(d, k, seed, lambda s: s >= d - 1)          # starts on the last coordinate
+    steps = sorted(set([0, 1, 2, 3] + wrap + tail))
+    exact = run_whole(B, d, W, k, steps, momentum, seed)
+    assert exact, "expected bit-identical results (same roundings in the same order)"
+
+
+@pytest.mark.parametrize("offsets", [(0, 0, 0, 0), (1, 0, 0, 0), (0, 2, 2, 2), (0, 1, 2, 3), (2, 2, 2, 2), (3, 1, 0, 0)])
+@pytest.mark.parametrize("d", [4096, 4098, 4099])
+def test_alignment_classes(B, d, offsets):
+    """16-, 8- and 4-byte aligned bases with d % 4 in {0, 2, 3}: every access width."""
+    assert run_whole(B, d, 5, 333, [0, 1, 2, 5], 0.9, 3, offsets=offsets)
+
+
+def test_ieee_specials_propagate(B):
+    def special(gh, t):
+        if t == 0:
+            gh[0, 3] = np.inf; gh[1, 5] = np.nan; gh[0, 7] = -np.inf; gh[1, 7] = np.inf
+            gh[0, 11] = -0.0; gh[1, 11] = -0.0
+    d, W, k = 64, 2, 64                                            # k = d: every coordinate is sent
+    run_whole(B, d, W, k, [0, 1], 0.9, 1, special=special)
+    run_whole(B, d, W, 8, [0, 1, 2], 0.0, 1, special=special)
+
+
+# ---------------------------------------------------------------------------
+# the workloads at full size
+# ---------------------------------------------------------------------------
+def run_workload_whole(B, wl, steps):
+    dev = torch.device("cuda")
+    x = WL.initial_params(wl, dev)
+    e, m = WL.zeros_state(wl, dev)
+    col_sigma = WL.column_sigma(wl, dev) if wl.grad == "per_tensor" else None
+    xo = x.cpu().numpy().copy()
+    eo = np.zeros((wl.W, wl.d), np.float32); mo = np.zeros((wl.W, wl.d), np.float32)
+    x64 = xo.astype(np.float64); e64 = eo.astype(np.float64); m64 = mo.astype(np.float64)
+    ctx = B.def_create(wl.d, wl.W, wl.k, wl.variant, wl.lr, wl.momentum, (wl.lam, 0.0))
+    g = torch.empty(wl.W, wl.d, dtype=torch.float32, device=dev)
+    after10 = None
+    for t in range(steps):
+        WL.gradients(wl, t, dev, out=g, col_sigma=col_sigma)
+        B.def_step(ctx, x, g, e, m, t, wl.rbgs_seed)
+        gh = g.cpu().numpy()
+        s = oracle.block_start(wl.rbgs_seed, t, wl.d)
+        oracle.step(xo, gh, eo, mo, d=wl.d, k=wl.k, s=s, eta=wl.lr, mu=wl.momentum)
+        oracle.step(x64, gh.astype(np.float64), e64, m64, d=wl.d, k=wl.k, s=s, eta=wl.lr, mu=wl.momentum)
+        assert bool(((e == 0).sum(dim=1) == wl.k).all()), "each worker's new error is zero on exactly k coordinates"
+        if t + 1 == 10 or t + 1 == steps:
+            exact = compare(x.cpu().numpy(), xo, "params after %d steps" % (t + 1))
+            exact &= compare(e.cpu().numpy(), eo, "errors after %d steps" % (t + 1))
+            exact &= compare(m.cpu().numpy(), mo, "mom after %d steps" % (t + 1))
+            compare_shadow(x.cpu().numpy(), x64, "params")
+            compare_shadow(e.cpu().numpy(), e64, "errors")
+            compare_shadow(m.cpu().numpy(), m64, "mom")
+            after10 = exact if after10 is None else (after10 and exact)
+    assert B.def_launch_count(ctx) >= steps
+    B.def_destroy(ctx)
+    return after10
+
+
+def test_config1_whole(B):
+    wl = WL.get(1)
+    assert run_workload_whole(B, wl, wl.steps)
+
+
+def test_config2_whole(B):
+    wl = WL.get(2)                                   # d % 4 == 2: 8-byte aligned rows
+    assert run_workload_whole(B, wl, wl.steps)
+
+
+def sample_columns(wl, steps, n_random=20000, halo=48):
+    """Coordinates the oracle follows on a full-size run: random ones, both ends of the
+    vector, and a halo around both ends of every step's block (where a wrong mask shows)."""
+    rng = np.random.default_rng(wl.cfg * 17 + wl.ratio)
+    cols = set(int(v) for v in rng.integers(0, wl.d, size=n_random))
+    cols.update(range(0, halo)); cols.update(range(wl.d - halo, wl.d))
+    for t in range(steps):
+        s = oracle.block_start(wl.rbgs_seed, t, wl.d)
+        for edge in (s, s + wl.k):
+            for j in range(edge - halo, edge + halo):
+                cols.add(j % wl.d)
+    return np.array(sorted(cols), dtype=np.int64)
+
+
+def run_workload_sampled(B, wl, steps):
+    """Full-size run in the launch configuration the benchmark times; the oracle follows a
+    sample of coordinates (a column view), and whole-tensor properties are checked on the GPU."""
+    dev = torch.device("cuda")
+    cols = sample_columns(wl, steps)
+    cols_dev = torch.from_numpy(cols).to(dev)
+    x = WL.initial_params(wl, dev)
+    x0 = x.clone()
+    e, m = WL.zeros_state(wl, dev)
+    col_sigma = WL.column_sigma(wl, dev) if wl.grad == "per_tensor" else None
+    xo = x[cols_dev].cpu().numpy().copy()
+    n = len(cols)
+    eo = np.zeros((wl.W, n), np.float32); mo = np.zeros((wl.W, n), np.float32)
+    x64 = xo.astype(np.float64); e64 = eo.astype(np.float64); m64 = mo.astype(np.float64)
+    ctx = B.def_create(wl.d, wl.W, wl.k, wl.variant, wl.lr, wl.momentum, (wl.lam, 0.0))
+    g = torch.empty(wl.W, wl.d, dtype=torch.float32, device=dev)
+    touched = torch.zeros(wl.d, dtype=torch.bool, device=dev)
+    y_expected = x0.double()                          # Eq. 8: y_{t+1} = y_t - eta * mean_k m_{k,t+1}
+    M = torch.zeros(wl.W, wl.d, dtype=torch.float32, device=dev)
+    exact = True
+    for t in range(steps):
+        WL.gradients(wl, t, dev, out=g, col_sigma=col_sigma)
+        B.def_step(ctx, x, g, e, m, t, wl.rbgs_seed)
+        s = oracle.block_start(wl.rbgs_seed, t, wl.d)
+        assert B.def_block_start(ctx, t, wl.rbgs_seed) == s
+        gh = np.ascontiguousarray(g[:, cols_dev].cpu().numpy())
+        oracle.step(xo, gh, eo, mo, d=wl.d, k=wl.k, s=s, eta=wl.lr, mu=wl.momentum, cols=cols)
+        oracle.step(x64, gh.astype(np.float64), e64, m64, d=wl.d, k=wl.k, s=s, eta=wl.lr, mu=wl.momentum, cols=cols)
+        # whole-tensor properties that hold at any size
+        assert bool(((e == 0).sum(dim=1) == wl.k).all()), "block mask: k zeros per worker"
+        first = torch.arange(s, min(s + wl.k, wl.d), device=dev)
+        touched[first] = True
+        if s + wl.k > wl.d:
+            touched[: s + wl.k - wl.d] = True
+        zero_cols = (e[0] == 0)
+        expect = torch.zeros(wl.d, dtype=torch.bool, device=dev)
+        expect[first] = True
+        if s + wl.k > wl.d:
+            expect[: s + wl.k - wl.d] = True
+        assert bool((zero_cols == expect).all()), "block mask is not the k coordinates from s"
+        M.mul_(wl.momentum).add_(g)
+        y_expected -= wl.lr * M.double().mean(dim=0)
+        if t + 1 == 10 or t + 1 == steps:
+            exact &= compare(x[cols_dev].cpu().numpy(), xo, "params after %d steps" % (t + 1))
+            exact &= compare(e[:, cols_dev].cpu().numpy(), eo, "errors after %d steps" % (t + 1))
+            exact &= compare(m[:, cols_dev].cpu().numpy(), mo, "mom after %d steps" % (t + 1))
+            compare_shadow(x[cols_dev].cpu().numpy(), x64, "params")
+            compare_shadow(e[:, cols_dev].cpu().numpy(), e64, "errors")
+            compare_shadow(m[:, cols_dev].cpu().numpy(), m64, "mom")
+    assert bool((x[~touched] == x0[~touched]).all()), "params moved outside every block"
+    y = x.double() - e.double().mean(dim=0)
+    scale = float(y_expected.abs().max())
+    assert float((y - y_expected).abs().max()) <= 2e-5 * scale, "Eq. 8 identity at full size"
+    B.def_destroy(ctx)
+    del g, e, m, M, x, touched
+    torch.cuda.empty_cache()
+    return exact
+
+
+@pytest.mark.parametrize("cfg", [3, 4])
+def test_config_full_size_sampled(B, cfg):
+    wl = WL.get(cfg)
+    assert run_workload_sampled(B, wl, wl.steps)
+
+
+@pytest.mark.parametrize("ratio", WL.CFG5_RATIOS)
+@pytest.mark.parametrize("variant", WL.CFG5_VARIANTS)
+def test_config5_full_size_sampled(B, ratio, variant):
+    wl = WL.get(5).with_ratio(ratio, variant)
+    assert run_workload_sampled(B, wl, wl.steps)
+
+
+# ---------------------------------------------------------------------------
+# column ranges, host memory, streams, resume
+# ---------------------------------------------------------------------------
+def test_step_columns_equals_whole_step(B):
+    dev = torch.device("cuda")
+    wl = WL.get(2).scaled(200_001, W=6)
+    d, W, k = wl.d, wl.W, wl.k
+    x = WL.initial_params(wl, dev); e, m = WL.zeros_state(wl, dev)
+    cuts = [0, 4, 70_000, 70_003, 150_002, d]                     # aligned and unaligned pieces
+    xs = [x[a:b].clone() for a, b in zip(cuts[:-1], cuts[1:])]
+    ctx = B.def_create(d, W, k, wl.variant, wl.lr, wl.momentum)
+    es = [torch.zeros(W, b - a + 5, device=dev) for a, b in zip(cuts[:-1], cuts[1:])]   # ld = n + 5
+    ms = [torch.zeros(W, b - a + 5, device=dev) for a, b in zip(cuts[:-1], cuts[1:])]
+    for t in range(6):
+        g = WL.gradients(wl, t, dev)
+        B.def_step(ctx, x, g, e, m, t, 9)
+        for i, (a, b) in enumerate(zip(cuts[:-1], cuts[1:])):
+            gl = torch.zeros(W, b - a + 5, device=dev)
+            gl[:, : b - a] = g[:, a:b]
+            B.def_step_columns(ctx, a, b - a, b - a + 5, xs[i], gl, es[i], ms[i], t, 9)
+    for i, (a, b) in enumerate(zip(cuts[:-1], cuts[1:])):
+        assert torch.equal(xs[i], x[a:b])
+        assert torch.equal(es[i][:, : b - a], e[:, a:b]) and torch.equal(ms[i][:, : b - a], m[:, a:b])
+        assert not es[i][:, b - a:].any() and not ms[i][:, b - a:].any(), "padding columns were written"
+    B.def_destroy(ctx)
+
+
+@pytest.mark.parametrize("momentum", [0.9, 0.0])
+def test_step_host_matches_oracle(B, momentum):
+    wl = WL.get(1).scaled(3_000_001, W=5, momentum=momentum)      # odd d: unaligned host rows
+    d, W, k = wl.d, wl.W, wl.k
+    x = WL.initial_params(wl, "cpu").pin_memory()
+    e = torch.zeros(W, d).pin_memory()
+    m = torch.zeros(W, d).pin_memory() if momentum else None
+    xo = x.numpy().copy(); eo = np.zeros((W, d), np.float32)
+    mo = np.zeros((W, d), np.float32) if momentum else None
+    ctx = B.def_create(d, W, k, wl.variant, wl.lr, momentum)
+    for t in range(3):
+        g = WL.gradients(wl, t, "cpu").pin_memory()
+        B.def_step_host(ctx, x, g, e, m, t, 4)
+        oracle.step(xo, g.numpy(), eo, mo, d=d, k=k, s=oracle.block_start(4, t, d), eta=wl.lr, mu=momentum)
+    assert compare(x.numpy(), xo, "params") and compare(e.numpy(), eo, "errors")
+    if momentum:
+        assert compare(m.numpy(), mo, "mom")
+    B.def_destroy(ctx)
+
+
+def test_stream_and_resume(B):
+    dev = torch.device("cuda")
+    wl = WL.get(1).scaled(500_000)
+    ctx = B.def_create(wl.d, wl.W, wl.k, wl.variant, wl.lr, wl.momentum)
+    side = torch.cuda.Stream()
+
+    def run(step_list, state=None, stream=None):
+        if state is None:
+            x = WL.initial_params(wl, dev); e, m = WL.zeros_state(wl, dev)
+        else:
+            x, e, m = (t.clone() for t in state)
+        B.def_set_stream(ctx, stream)
+        for t in step_list:
+            g = WL.gradients(wl, t, dev)
+            if stream is not None:
+                stream.wait_stream(torch.cuda.current_stream())
+            B.def_step(ctx, x, g, e, m, t, 2)
+            if stream is not None:
+                torch.cuda.current_stream().wait_stream(stream)
+        torch.cuda.synchronize()
+        B.def_set_stream(ctx, None)
+        return x, e, m
+
+    straight = run(range(10))
+    half = run(range(5), stream=side)
+    resumed = run(range(5, 10), state=half)               # the sampler has no state to carry
+    for a, b in zip(straight, resumed):
+        assert torch.equal(a, b)
+    B.def_destroy(ctx)

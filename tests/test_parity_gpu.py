@@ -136,11 +136,13 @@ def run_whole(B, d, W, k, steps, momentum, seed, lr=0.1, offsets=(0, 0, 0, 0), s
         assert B.def_block_start(ctx, t, seed) == s
         oracle.step(xo, gh, eo, mo, d=d, k=k, s=s, eta=lr, mu=momentum)
         oracle.step(x64, gh.astype(np.float64), e64, m64, d=d, k=k, s=s, eta=lr, mu=momentum)
-        # the mask, bit-exact: after a step e' is +0 exactly on the block
+        # the mask, bit-exact: e' is +0 on the block, and nowhere the oracle's is not
         mask = oracle.block_mask(d, k, s)
         eg = e.cpu().numpy()
         if special is None:
-            assert np.array_equal(eg == 0, np.broadcast_to(mask, (W, d))), "block mask differs at step %d" % t
+            assert not eg[:, mask].any() and not np.signbit(eg[:, mask]).any(), "block not zeroed at step %d" % t
+            assert np.array_equal(eg == 0, eo == 0), "zero pattern of the new error differs at step %d" % t
+            assert np.count_nonzero(eg[:, ~mask] == 0) <= 2, "coordinates outside the block were zeroed"
         assert np.array_equal(g.cpu().numpy(), gh, equal_nan=True), "grads must not be written"
     torch.cuda.synchronize()
     for chk in (cx, cg, ce, cm):
@@ -215,7 +217,9 @@ def run_workload_whole(B, wl, steps):
         s = oracle.block_start(wl.rbgs_seed, t, wl.d)
         oracle.step(xo, gh, eo, mo, d=wl.d, k=wl.k, s=s, eta=wl.lr, mu=wl.momentum)
         oracle.step(x64, gh.astype(np.float64), e64, m64, d=wl.d, k=wl.k, s=s, eta=wl.lr, mu=wl.momentum)
-        assert bool(((e == 0).sum(dim=1) == wl.k).all()), "each worker's new error is zero on exactly k coordinates"
+        zeros = (e == 0).sum(dim=1)          # k per worker, plus the rare p that is exactly 0
+        assert bool((zeros >= wl.k).all()) and int(zeros.sum()) - wl.W * wl.k <= 8 + wl.W * wl.d // 10 ** 6
+        assert np.array_equal(e.cpu().numpy() == 0, eo == 0), "zero pattern of the new error differs"
         if t + 1 == 10 or t + 1 == steps:
             exact = compare(x.cpu().numpy(), xo, "params after %d steps" % (t + 1))
             exact &= compare(e.cpu().numpy(), eo, "errors after %d steps" % (t + 1))
@@ -282,19 +286,20 @@ def run_workload_sampled(B, wl, steps):
         oracle.step(xo, gh, eo, mo, d=wl.d, k=wl.k, s=s, eta=wl.lr, mu=wl.momentum, cols=cols)
         oracle.step(x64, gh.astype(np.float64), e64, m64, d=wl.d, k=wl.k, s=s, eta=wl.lr, mu=wl.momentum, cols=cols)
         # whole-tensor properties that hold at any size
-        assert bool(((e == 0).sum(dim=1) == wl.k).all()), "block mask: k zeros per worker"
-        first = torch.arange(s, min(s + wl.k, wl.d), device=dev)
-        touched[first] = True
-        if s + wl.k > wl.d:
-            touched[: s + wl.k - wl.d] = True
-        zero_cols = (e[0] == 0)
-        expect = torch.zeros(wl.d, dtype=torch.bool, device=dev)
-        expect[first] = True
+        expect = torch.zeros(wl.d, dtype=torch.bool, device=dev)        # the k coordinates from s
+        expect[s:min(s + wl.k, wl.d)] = True
         if s + wl.k > wl.d:
             expect[: s + wl.k - wl.d] = True
-        assert bool((zero_cols == expect).all()), "block mask is not the k coordinates from s"
+        assert int(expect.sum()) == wl.k
+        touched |= expect
+        is_zero = (e == 0)
+        assert bool(is_zero[:, expect].all()), "a block coordinate kept a non-zero error"
+        # outside the block e' = p, which is exactly 0 only where a drawn gradient is (a few in 1e8)
+        stray = int(is_zero.sum()) - wl.W * wl.k
+        assert 0 <= stray <= 8 + wl.W * wl.d // 10 ** 6, "coordinates outside the block were zeroed: %d" % stray
+        del is_zero
         M.mul_(wl.momentum).add_(g)
-        y_expected -= wl.lr * M.double().mean(dim=0)
+        y_expected -= wl.lr * (M.sum(dim=0, dtype=torch.float64) / wl.W)
         if t + 1 == 10 or t + 1 == steps:
             exact &= compare(x[cols_dev].cpu().numpy(), xo, "params after %d steps" % (t + 1))
             exact &= compare(e[:, cols_dev].cpu().numpy(), eo, "errors after %d steps" % (t + 1))
@@ -303,7 +308,7 @@ def run_workload_sampled(B, wl, steps):
             compare_shadow(e[:, cols_dev].cpu().numpy(), e64, "errors")
             compare_shadow(m[:, cols_dev].cpu().numpy(), m64, "mom")
     assert bool((x[~touched] == x0[~touched]).all()), "params moved outside every block"
-    y = x.double() - e.double().mean(dim=0)
+    y = x.double() - e.sum(dim=0, dtype=torch.float64) / wl.W
     scale = float(y_expected.abs().max())
     assert float((y - y_expected).abs().max()) <= 2e-5 * scale, "Eq. 8 identity at full size"
     B.def_destroy(ctx)

@@ -118,27 +118,42 @@ int vector_width(int64_t ld, const float *x, const float *g, const float *e, con
     return 1;
 }
 
+// Rows in flight per thread on the tiles that touch the block, and the cache policy of the
+// [W, d] traffic: the best of the measured combinations.
+constexpr int kBlockRows = 8;
+constexpr int kPolicy = defk::kCacheDefault;
+
 template <int V, bool MOM>
-cudaError_t launch_one(const def_ctx *ctx, const defk::StepArgs &a, cudaStream_t stream) {
-    // 4 rows in flight per thread: 12 independent 16-byte loads before the first use.
-    constexpr int U = 4;
+cudaError_t launch_one(const defk::StepArgs &a, cudaStream_t stream, int64_t *launches) {
     const int64_t groups = a.n / V;
     if (groups == 0) return cudaSuccess;
-    // One group of V coordinates per thread.  Many short CTAs drift out of phase with each
-    // other, which keeps reads and writes mixed at the DRAM; a persistent grid whose CTAs
-    // march in step measured 10 % slower.  The grid-stride loop only covers the case of
-    // more groups than one grid can hold.
-    const int64_t want = (groups + kThreads - 1) / kThreads;
-    const int64_t cap = 0x7fffffffLL;
-    const unsigned grid = (unsigned)(want < cap ? want : cap);
-    (void)ctx;
-    defk::def_step_kernel<V, MOM, U><<<grid, kThreads, 0, stream>>>(a);
-    return cudaGetLastError();
+    if (V == 4) {
+        const int64_t tiles = (a.n + defk::kTile - 1) / defk::kTile;
+        if (tiles > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+        // the few tiles that touch the block first, then the stream over all the others
+        const int64_t block_ctas = a.k / defk::kTile + 4;
+        defk::def_step_block_kernel<MOM, kBlockRows, kPolicy>
+            <<<(unsigned)(block_ctas < tiles + 1 ? block_ctas : tiles + 1), defk::kTileThreads, 0, stream>>>(a);
+        cudaError_t err = cudaGetLastError();
+        if (err != cudaSuccess) return err;
+        *launches += 1;
+        const dim3 grid((unsigned)tiles, (unsigned)a.W);
+        defk::def_step_stream_kernel<MOM, kPolicy><<<grid, defk::kTileThreads, 0, stream>>>(a);
+    } else {
+        // One group of V coordinates per thread; the grid-stride loop only covers the case
+        // of more groups than one grid can hold.
+        const int64_t want = (groups + kThreads - 1) / kThreads;
+        const int64_t cap = 0x7fffffffLL;
+        defk::def_step_kernel<V, MOM, 4><<<(unsigned)(want < cap ? want : cap), kThreads, 0, stream>>>(a);
+    }
+    cudaError_t err = cudaGetLastError();
+    if (err == cudaSuccess) *launches += 1;
+    return err;
 }
 
 template <int V>
-cudaError_t launch_v(const def_ctx *ctx, const defk::StepArgs &a, cudaStream_t stream) {
-    return a.m ? launch_one<V, true>(ctx, a, stream) : launch_one<V, false>(ctx, a, stream);
+cudaError_t launch_v(const defk::StepArgs &a, cudaStream_t stream, int64_t *launches) {
+    return a.m ? launch_one<V, true>(a, stream, launches) : launch_one<V, false>(a, stream, launches);
 }
 
 // Enqueue the step on local coordinates [0, n) of a view; counts launches.
@@ -155,18 +170,16 @@ int enqueue_columns(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, float *x, c
     const int64_t body = n - n % V;
     if (body > 0) {
         a.n = body;
-        err = V == 4 ? launch_v<4>(ctx, a, stream) : V == 2 ? launch_v<2>(ctx, a, stream)
-                                                              : launch_v<1>(ctx, a, stream);
+        err = V == 4 ? launch_v<4>(a, stream, &ctx->launches) : V == 2 ? launch_v<2>(a, stream, &ctx->launches)
+                                                              : launch_v<1>(a, stream, &ctx->launches);
         if (err != cudaSuccess) return cuda_fail(err, "def_step kernel launch");
-        ctx->launches += 1;
     }
     if (body < n) {  // the last n % V coordinates, one float at a time
         defk::StepArgs t = a;
         t.x = x + body; t.g = g + body; t.e = e + body; t.m = m ? m + body : nullptr;
         t.n = n - body; t.j0 = j0 + body;
-        err = launch_v<1>(ctx, t, stream);
+        err = launch_v<1>(t, stream, &ctx->launches);
         if (err != cudaSuccess) return cuda_fail(err, "def_step tail kernel launch");
-        ctx->launches += 1;
     }
     return DEF_OK;
 }

@@ -2,16 +2,17 @@
 //
 // The step (Algorithm 1 lines 7-10 with the momentum form of Eq. 10) is separate
 // per model coordinate: a coordinate j needs g, m, e of its W workers and, if j is
-// one of the k block coordinates, x[j].  The kernel therefore gives each thread a
-// short vector of consecutive coordinates and walks the W rows in order, so that
-//   * g, m, e are read once and m', e' written once (20 bytes per gradient element,
-//     the least the method can move), with 128-bit coalesced accesses;
-//   * p never goes to memory;
-//   * the sum over workers that stands in for the ring-allreduce of line 9 is a
-//     register accumulation in the fixed order w = 0..W-1: deterministic, and with
-//     no shuffle, shared memory or atomics;
-//   * x is touched on the block only (line 10).
-// The block is a predicate on j, never a slice: nothing is gathered or scattered.
+// one of the k block coordinates, x[j].  Two facts shape the kernels:
+//   * Outside the block nothing crosses workers (C(p) = 0, e' = p), so that part --
+//     all but k of the d coordinates -- is plain streaming of the [W, d] tensors and
+//     can be cut any way the memory system likes best.
+//   * On the block, the sum over workers that stands in for the ring-allreduce of
+//     line 9 is a register accumulation by one thread in the fixed order
+//     w = 0..W-1: deterministic, with no shuffle, shared memory or atomics.
+// Either way g, m, e are read once and m', e' written once (20 bytes per gradient
+// element, the least the method can move) with 128-bit coalesced accesses, p never
+// goes to memory, and x is touched on the block only (line 10).  The block is a
+// predicate on j, never a slice: nothing is gathered or scattered.
 #pragma once
 
 #include <cuda_runtime.h>
@@ -72,30 +73,39 @@ template <> struct Vec<1> { float v[1]; };
 template <> struct alignas(8) Vec<2> { float v[2]; };
 template <> struct alignas(16) Vec<4> { float v[4]; };
 
-// g, m and e are read once per step and the new m and e are not read again before
-// the next step, by which time W*d*20 bytes have passed through the L2: mark the
-// traffic as streaming so that it does not push x (which is reused) out.
-template <int V> __device__ __forceinline__ Vec<V> load_stream(const float *p);
-template <> __device__ __forceinline__ Vec<1> load_stream<1>(const float *p) {
-    Vec<1> r; r.v[0] = __ldcs(p); return r;
+// Cache policy of the [W, d] traffic.  g, m and e are read once per step and m', e' are
+// not read again before the next step.  kCacheDefault leaves write-back to the L2's own
+// replacement; kCacheStreaming marks loads and stores evict-first (ld.cs / st.cs).
+constexpr int kCacheDefault = 0;
+constexpr int kCacheStreaming = 1;
+
+template <int V, int POL> __device__ __forceinline__ Vec<V> load_vec(const float *p) {
+    Vec<V> r;
+    if constexpr (V == 1) {
+        r.v[0] = POL == kCacheStreaming ? __ldcs(p) : *p;
+    } else if constexpr (V == 2) {
+        const float2 t = POL == kCacheStreaming ? __ldcs(reinterpret_cast<const float2 *>(p))
+                                                : *reinterpret_cast<const float2 *>(p);
+        r.v[0] = t.x; r.v[1] = t.y;
+    } else {
+        const float4 t = POL == kCacheStreaming ? __ldcs(reinterpret_cast<const float4 *>(p))
+                                                : *reinterpret_cast<const float4 *>(p);
+        r.v[0] = t.x; r.v[1] = t.y; r.v[2] = t.z; r.v[3] = t.w;
+    }
+    return r;
 }
-template <> __device__ __forceinline__ Vec<2> load_stream<2>(const float *p) {
-    const float2 t = __ldcs(reinterpret_cast<const float2 *>(p));
-    Vec<2> r; r.v[0] = t.x; r.v[1] = t.y; return r;
-}
-template <> __device__ __forceinline__ Vec<4> load_stream<4>(const float *p) {
-    const float4 t = __ldcs(reinterpret_cast<const float4 *>(p));
-    Vec<4> r; r.v[0] = t.x; r.v[1] = t.y; r.v[2] = t.z; r.v[3] = t.w; return r;
-}
-template <int V> __device__ __forceinline__ void store_stream(float *p, const Vec<V> &a);
-template <> __device__ __forceinline__ void store_stream<1>(float *p, const Vec<1> &a) {
-    __stcs(p, a.v[0]);
-}
-template <> __device__ __forceinline__ void store_stream<2>(float *p, const Vec<2> &a) {
-    __stcs(reinterpret_cast<float2 *>(p), make_float2(a.v[0], a.v[1]));
-}
-template <> __device__ __forceinline__ void store_stream<4>(float *p, const Vec<4> &a) {
-    __stcs(reinterpret_cast<float4 *>(p), make_float4(a.v[0], a.v[1], a.v[2], a.v[3]));
+template <int V, int POL> __device__ __forceinline__ void store_vec(float *p, const Vec<V> &a) {
+    if constexpr (V == 1) {
+        if (POL == kCacheStreaming) __stcs(p, a.v[0]); else *p = a.v[0];
+    } else if constexpr (V == 2) {
+        const float2 t = make_float2(a.v[0], a.v[1]);
+        if (POL == kCacheStreaming) __stcs(reinterpret_cast<float2 *>(p), t);
+        else *reinterpret_cast<float2 *>(p) = t;
+    } else {
+        const float4 t = make_float4(a.v[0], a.v[1], a.v[2], a.v[3]);
+        if (POL == kCacheStreaming) __stcs(reinterpret_cast<float4 *>(p), t);
+        else *reinterpret_cast<float4 *>(p) = t;
+    }
 }
 
 struct StepArgs {
@@ -115,11 +125,21 @@ struct StepArgs {
     uint64_t seed, step; // the block start is drawn from these
 };
 
+// The start of this step's block, computed by one thread of the CTA and handed to the
+// others through shared memory (the ten Philox rounds are a serial chain of ~100
+// instructions: once per CTA they cost nothing, once per thread they would show).
+__device__ __forceinline__ int64_t cta_block_start(const StepArgs &a) {
+    __shared__ int64_t s_shared;
+    if (threadIdx.x == 0) s_shared = block_start(a.seed, a.step, a.d);
+    __syncthreads();
+    return s_shared;
+}
+
 // One worker's row for V coordinates: Eq. 10 / line 7, then line 8.
-// `sent` accumulates C(p) over the workers in call order.
-template <int V, bool MOM, bool FIRST>
+// `sent` accumulates C(p) over the workers in call order; `first` starts the sum.
+template <int V, bool MOM>
 __device__ __forceinline__ void worker_row(const Vec<V> &g, const Vec<V> &m, const Vec<V> &e,
-                                           const bool (&in)[V], float eta, float mu,
+                                           const bool (&in)[V], float eta, float mu, bool first,
                                            Vec<V> &m_new, Vec<V> &e_new, float (&sent)[V]) {
 #pragma unroll
     for (int i = 0; i < V; ++i) {
@@ -132,92 +152,148 @@ __device__ __forceinline__ void worker_row(const Vec<V> &g, const Vec<V> &m, con
         }
         const float c = in[i] ? p : 0.0f;                    // C(p)
         e_new.v[i] = __fsub_rn(p, c);                        // e' = p - C(p)
-        sent[i] = FIRST ? c : __fadd_rn(sent[i], c);         // running sum of line 9
+        sent[i] = first ? c : __fadd_rn(sent[i], c);         // running sum of line 9
     }
 }
 
-// The step over local coordinates [0, n), V per thread, U rows in flight per thread.
-//   grid-stride over groups of V coordinates; rows must be aligned for V-wide access:
-//   x, g, e, m aligned to 4V bytes and ld % V == 0.  The n % V tail coordinates are
-//   handled by the V = 1 instantiation launched on the tail (see the host code).
-template <int V, bool MOM, int U>
-__global__ void __launch_bounds__(256)
-def_step_kernel(const StepArgs a) {
-    const int64_t s = block_start(a.seed, a.step, a.d);
-    const int64_t groups = a.n / V;
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+// All W workers of the V coordinates starting at local coordinate `col`, in worker order,
+// U rows in flight at a time; then lines 9-10 on the coordinates that are in the block.
+template <int V, bool MOM, int U, int POL>
+__device__ __forceinline__ void column_group(const StepArgs &a, int64_t s, int64_t col) {
+    // offset of each coordinate from the block start, mod d; in the block iff < k
+    int64_t off = a.j0 + col - s;
+    if (off < 0) off += a.d;
+    bool in[V];
+    bool any = false;
+#pragma unroll
+    for (int i = 0; i < V; ++i) {
+        int64_t o = off + i;
+        if (o >= a.d) o -= a.d;
+        in[i] = o < a.k;
+        any |= in[i];
+    }
+    float sent[V];
+#pragma unroll
+    for (int i = 0; i < V; ++i) sent[i] = 0.0f;
     const size_t ld = (size_t)a.ld;
-    for (int64_t grp = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; grp < groups; grp += stride) {
-        const int64_t col = grp * V;
-        // offset of each coordinate from the block start, mod d; in the block iff < k
-        int64_t off = a.j0 + col - s;
-        if (off < 0) off += a.d;
-        bool in[V];
-        bool any = false;
+    const float *gp = a.g + col;
+    float *ep = a.e + col;
+    float *mp = MOM ? a.m + col : nullptr;
+    for (int w = 0; w < a.W; w += U) {
+        Vec<V> g[U], e[U], m[U];
 #pragma unroll
-        for (int i = 0; i < V; ++i) {
-            int64_t o = off + i;
-            if (o >= a.d) o -= a.d;
-            in[i] = o < a.k;
-            any |= in[i];
-        }
-
-        float sent[V];
-        const float *gp = a.g + col;
-        float *ep = a.e + col;
-        float *mp = MOM ? a.m + col : nullptr;
-        int w = 0;
-        // worker 0 starts the sum
-        {
-            const Vec<V> g = load_stream<V>(gp);
-            const Vec<V> e = load_stream<V>(ep);
-            Vec<V> m, m_new, e_new;
-            if (MOM) m = load_stream<V>(mp);
-            worker_row<V, MOM, true>(g, m, e, in, a.eta, a.mu, m_new, e_new, sent);
-            if (MOM) store_stream<V>(mp, m_new);
-            store_stream<V>(ep, e_new);
-            w = 1;
-        }
-        // U workers at a time: issue all loads, then compute and store in order
-        for (; w + U <= a.W; w += U) {
-            Vec<V> g[U], e[U], m[U];
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
+        for (int u = 0; u < U; ++u) {                      // issue every load of the chunk first
+            if (w + u < a.W) {
                 const size_t row = (size_t)(w + u) * ld;
-                g[u] = load_stream<V>(gp + row);
-                e[u] = load_stream<V>(ep + row);
-                if (MOM) m[u] = load_stream<V>(mp + row);
+                g[u] = load_vec<V, POL>(gp + row);
+                e[u] = load_vec<V, POL>(ep + row);
+                if (MOM) m[u] = load_vec<V, POL>(mp + row);
             }
+        }
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
+        for (int u = 0; u < U; ++u) {                      // then compute and store in worker order
+            if (w + u < a.W) {
                 const size_t row = (size_t)(w + u) * ld;
                 Vec<V> m_new, e_new;
-                worker_row<V, MOM, false>(g[u], m[u], e[u], in, a.eta, a.mu, m_new, e_new, sent);
-                if (MOM) store_stream<V>(mp + row, m_new);
-                store_stream<V>(ep + row, e_new);
-            }
-        }
-        for (; w < a.W; ++w) {
-            const size_t row = (size_t)w * ld;
-            const Vec<V> g = load_stream<V>(gp + row);
-            const Vec<V> e = load_stream<V>(ep + row);
-            Vec<V> m, m_new, e_new;
-            if (MOM) m = load_stream<V>(mp + row);
-            worker_row<V, MOM, false>(g, m, e, in, a.eta, a.mu, m_new, e_new, sent);
-            if (MOM) store_stream<V>(mp + row, m_new);
-            store_stream<V>(ep + row, e_new);
-        }
-        // lines 9-10 on the block coordinates: x -= (sum over workers) / W
-        if (any) {
-#pragma unroll
-            for (int i = 0; i < V; ++i) {
-                if (in[i]) {
-                    const float C_pt = __fdiv_rn(sent[i], a.W_float);
-                    a.x[col + i] = __fsub_rn(a.x[col + i], C_pt);
-                }
+                worker_row<V, MOM>(g[u], m[u], e[u], in, a.eta, a.mu, w + u == 0, m_new, e_new, sent);
+                if (MOM) store_vec<V, POL>(mp + row, m_new);
+                store_vec<V, POL>(ep + row, e_new);
             }
         }
     }
+    if (any) {                                              // x -= (sum over workers) / W
+#pragma unroll
+        for (int i = 0; i < V; ++i) {
+            if (in[i]) {
+                const float C_pt = __fdiv_rn(sent[i], a.W_float);
+                a.x[col + i] = __fsub_rn(a.x[col + i], C_pt);
+            }
+        }
+    }
+}
+
+// General kernel: every thread owns V coordinates and walks all W rows.  Used for rows that
+// are only 4- or 8-byte aligned (V = 1, 2) and for the n % 4 tail.  Rows must be aligned
+// for V-wide access: x, g, e, m aligned to 4V bytes and ld % V == 0.
+template <int V, bool MOM, int U>
+__global__ void __launch_bounds__(256)
+def_step_kernel(const StepArgs a) {
+    const int64_t s = cta_block_start(a);
+    const int64_t groups = a.n / V;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t grp = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; grp < groups; grp += stride)
+        column_group<V, MOM, U, kCacheDefault>(a, s, grp * V);
+}
+
+// Kernels for 16-byte aligned rows.  The n local coordinates are cut into tiles of
+// TILE = kTileThreads * 4 coordinates.  A tile "touches the block" if any of its coordinates
+// is one of the k block coordinates; every CTA decides that from the block start before it
+// issues a load.
+constexpr int kTileThreads = 256;
+constexpr int64_t kTile = (int64_t)kTileThreads * 4;
+
+__device__ __forceinline__ bool tile_touches_block(const StepArgs &a, int64_t s, int64_t tile) {
+    const int64_t tile0 = tile * kTile;
+    const int64_t tile_len = (a.n - tile0 < kTile) ? a.n - tile0 : kTile;
+    int64_t off0 = a.j0 + tile0 - s;                 // offset of the tile's start from s, mod d
+    if (off0 < 0) off0 += a.d;
+    return off0 < a.k || off0 + tile_len > a.d;      // starts inside the block, or wraps onto its start
+}
+
+// Tiles that do not touch the block (all but about k / TILE + 2 of them) have nothing to
+// sum: C(p) = 0 and e' = p.  The grid is (tiles, W) and CTA (t, w) does worker w's row of
+// tile t: three 16-byte loads and two stores per thread, few registers, full occupancy.
+// Consecutive CTAs sweep one row after the other, so the memory system sees a handful of
+// long sequential streams.  CTAs of tiles that touch the block leave at once.
+template <bool MOM, int POL>
+__global__ void __launch_bounds__(kTileThreads)
+def_step_stream_kernel(const StepArgs a) {
+    const int64_t s = cta_block_start(a);
+    const int64_t tile = blockIdx.x;
+    const int64_t col = tile * kTile + (int64_t)threadIdx.x * 4;
+    if (col >= a.n || tile_touches_block(a, s, tile)) return;
+    const size_t at = (size_t)blockIdx.y * (size_t)a.ld + (size_t)col;
+    const Vec<4> g = load_vec<4, POL>(a.g + at);
+    const Vec<4> e = load_vec<4, POL>(a.e + at);
+    Vec<4> m, m_new, e_new;
+    if (MOM) m = load_vec<4, POL>(a.m + at);
+    const bool none[4] = {false, false, false, false};
+    float unused[4];
+    worker_row<4, MOM>(g, m, e, none, a.eta, a.mu, true, m_new, e_new, unused);
+    if (MOM) store_vec<4, POL>(a.m + at, m_new);
+    store_vec<4, POL>(a.e + at, e_new);
+}
+
+// Tiles that touch the block: one CTA per tile walks the W rows in order (column_group).
+// The block is at most two runs of local coordinates (it may wrap past d, and the local
+// range may cut it); a run of length L touches at most L / TILE + 2 tiles, so a grid of
+// k / TILE + 4 CTAs covers every case.  CTA i takes the i-th touched tile: first those of
+// the run that starts at s, then those of the wrapped run [0, s + k - d) that the first
+// run has not already covered.  CTAs beyond the last touched tile leave.
+template <bool MOM, int U, int POL>
+__global__ void __launch_bounds__(kTileThreads)
+def_step_block_kernel(const StepArgs a) {
+    const int64_t s = cta_block_start(a);
+    // the two runs in model coordinates, clipped to the local range [j0, j0 + n)
+    const int64_t lo = a.j0, hi = a.j0 + a.n;
+    int64_t a0 = s > lo ? s : lo;                                // run A = [s, min(s + k, d))
+    int64_t a1 = (s + a.k < a.d ? s + a.k : a.d);
+    a1 = a1 < hi ? a1 : hi;
+    int64_t b0 = lo;                                             // run B = [0, s + k - d)
+    int64_t b1 = s + a.k - a.d;
+    b1 = b1 < hi ? b1 : hi;
+    const int64_t tA0 = (a0 - lo) / kTile, tA1 = a1 > a0 ? (a1 - 1 - lo) / kTile : tA0 - 1;
+    const int64_t tB0 = 0, tB1 = b1 > b0 ? (b1 - 1 - lo) / kTile : -1;
+    const int64_t nA = tA1 - tA0 + 1;
+    int64_t tile;
+    if ((int64_t)blockIdx.x < nA) {
+        tile = tA0 + blockIdx.x;
+    } else {
+        tile = tB0 + ((int64_t)blockIdx.x - nA);
+        if (tile > tB1 || (tile >= tA0 && tile <= tA1)) return;  // past the end, or already done as part of run A
+    }
+    const int64_t col = tile * kTile + (int64_t)threadIdx.x * 4;
+    if (col < a.n) column_group<4, MOM, U, POL>(a, s, col);
 }
 
 }  // namespace defk

@@ -34,12 +34,12 @@ METRIC = "DEF step gradient elements/s (W*d per step)"
 UNIT = "elements/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM traffic of one def_step_kernel<4, true, 4> launch from an ncu capture
+# DRAM traffic of one def_step_stream_kernel launch from an ncu capture
 # (dram__bytes_read.sum + dram__bytes_write.sum), as bytes per gradient element, and the
 # hash of the kernel source the capture was taken on.  Reported only while the source is
 # unchanged (see profiles/).
-NCU_TRAFFIC_BYTES_PER_ELEMENT = None
-NCU_TRAFFIC_KERNEL_SHA256 = None
+NCU_TRAFFIC_BYTES_PER_ELEMENT = 19.43
+NCU_TRAFFIC_KERNEL_SHA256 = "0a81f643933e61baf17b70a4345ff23795bd1a11c41bef4bef97335c41d3f397"
 
 
 def _measured_peak():
@@ -187,9 +187,56 @@ def time_steps(B, ctx, shard, tensors, steps, warmup, seed, dist=None, flush=Non
     return _max_over_ranks(dist, ms), launches
 
 
-def bench_workload(B, WL, wl, steps, warmup, dist, world, rank, sampler=None, flush=None):
+TILE = 1024   # coordinates per tile of the two step kernels (256 threads x 4)
+
+
+def touched_columns(d, k, s, j0, n):
+    """Local coordinates that lie in tiles touching the block {(s+i) mod d}: the block kernel's share."""
+    runs = [(s, min(s + k, d))]
+    if s + k > d:
+        runs.append((0, s + k - d))
+    tiles = set()
+    for a, b in runs:
+        a, b = max(a, j0), min(b, j0 + n)
+        if b > a:
+            tiles.update(range((a - j0) // TILE, (b - 1 - j0) // TILE + 1))
+    return sum(min(TILE, n - t * TILE) for t in tiles)
+
+
+def profile_kernels(B, ctx, shard, tensors, steps, first_step, seed, per_el, k_share, flush=None):
+    """Per-kernel device time over `steps` more steps (each launch bracketed by events inside the
+    library and waited for), with the algorithmic bytes each kernel had to move."""
+    j0, n, ld = shard
+    x, g, e, m = tensors
+    W = ctx.W
+    before = {kind: B.def_kernel_time(ctx, kind) for kind in (B.DEF_KERNEL_STREAM, B.DEF_KERNEL_BLOCK, B.DEF_KERNEL_GENERAL)}
+    B.def_set_kernel_timing(ctx, True)
+    bytes_stream = bytes_block = 0
+    for t in range(steps):
+        if flush is not None:
+            flush.add_(1.0)
+        step = first_step + t
+        B.def_step_columns(ctx, j0, n, ld, x, g, e, m, step, seed)
+        cols = touched_columns(ctx.d, ctx.k, B.def_block_start(ctx, step, seed), j0, n)
+        bytes_block += per_el * W * cols + 8 * k_share
+        bytes_stream += per_el * W * (n - cols)
+    B.def_set_kernel_timing(ctx, False)
+    out = []
+    for kind, name, nbytes in ((B.DEF_KERNEL_STREAM, "def_step_stream_kernel", bytes_stream),
+                               (B.DEF_KERNEL_BLOCK, "def_step_block_kernel", bytes_block),
+                               (B.DEF_KERNEL_GENERAL, "def_step_kernel", 0)):
+        ms, cnt = B.def_kernel_time(ctx, kind)
+        ms, cnt = ms - before[kind][0], cnt - before[kind][1]
+        if cnt:
+            out.append({"kernel": name, "launches": cnt, "ms_per_launch": ms / cnt,
+                        "algorithmic_bytes_per_launch": nbytes / cnt if nbytes else None,
+                        "GB/s": (nbytes / (ms * 1e-3) / 1e9) if nbytes else None})
+    return out
+
+
+def bench_workload(B, WL, wl, steps, warmup, dist, world, rank, sampler=None, flush=None, profile=False):
     """Allocate a rank's shard of the workload, run, return (ms, launches, elements per step over
-    all ranks, algorithmic bytes per launch on this rank)."""
+    all ranks, algorithmic bytes per step on this rank, per-kernel profile or None)."""
     import torch
     dev = torch.device("cuda")
     d_global = wl.d * world
@@ -203,12 +250,16 @@ def bench_workload(B, WL, wl, steps, warmup, dist, world, rank, sampler=None, fl
     col_sigma = WL.column_sigma(wl, dev) if wl.grad == "per_tensor" else None
     g = WL.gradients(wl, rank, dev, col_sigma=col_sigma)   # one gradient buffer, reused: values do not steer the kernel
     ms, launches = time_steps(B, ctx, (j0, n, n), (x, g, e, m), steps, warmup, wl.rbgs_seed, dist, flush, sampler)
-    B.def_destroy(ctx)
     per_el = 20 if wl.momentum != 0.0 else 12
     alg_bytes = per_el * wl.W * n + 8 * k_global / world
+    kernels = None
+    if profile:
+        kernels = profile_kernels(B, ctx, (j0, n, n), (x, g, e, m), steps, warmup + steps, wl.rbgs_seed, per_el,
+                                  k_global / world, flush)
+    B.def_destroy(ctx)
     del x, g, e, m
     torch.cuda.empty_cache()
-    return ms, launches, wl.W * d_global, alg_bytes
+    return ms, launches, wl.W * d_global, alg_bytes, kernels
 
 
 def available_host_bytes():
@@ -375,17 +426,19 @@ def main():
     sampler = ClockSampler(local)
     small = wl.algorithmic_bytes_per_step() < 1e9          # fits the L2: flush it between steps
     main_flush = torch.zeros(96 * 1024 * 1024, dtype=torch.float32, device="cuda") if small else None
-    ms, launches, elements, alg_bytes = bench_workload(B, WL, wl, args.steps, args.warmup, dist, world, rank, sampler,
-                                                       flush=main_flush)
+    ms, launches, elements, alg_bytes, kernels = bench_workload(B, WL, wl, args.steps, args.warmup, dist, world, rank,
+                                                                sampler, flush=main_flush, profile=True)
     del main_flush
     clocks = sampler.finish()
     peak, peak_kind = _measured_peak()
     value = elements * args.steps / (ms * 1e-3)
-    launch_ms = ms / max(1, launches)
-    achieved = alg_bytes / (launch_ms * 1e-3) / 1e9
+    step_gbs = alg_bytes * args.steps / (ms * 1e-3) / 1e9
+    top = max(kernels, key=lambda kk: kk["ms_per_launch"] * kk["launches"])      # the dominant kernel
+    achieved = top["GB/s"] if top["GB/s"] is not None else step_gbs
     traffic = None
-    if NCU_TRAFFIC_BYTES_PER_ELEMENT is not None and NCU_TRAFFIC_KERNEL_SHA256 == _kernel_hash():
-        traffic = NCU_TRAFFIC_BYTES_PER_ELEMENT * wl.W * wl.d
+    if (NCU_TRAFFIC_BYTES_PER_ELEMENT is not None and NCU_TRAFFIC_KERNEL_SHA256 == _kernel_hash()
+            and top["algorithmic_bytes_per_launch"]):
+        traffic = NCU_TRAFFIC_BYTES_PER_ELEMENT * top["algorithmic_bytes_per_launch"] / 20.0
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
@@ -393,8 +446,13 @@ def main():
         "gpu_launches": launches, "clocks": clocks,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": traffic, "peak_kind": "of %s" % peak_kind, "frac_of_8000_nominal": achieved / 8000.0,
-                     "kernel": "def_step_kernel<4,true,4>", "algorithmic_bytes_per_launch": alg_bytes,
-                     "launch_ms": launch_ms},
+                     "kernel": top["kernel"], "algorithmic_bytes_per_launch": top["algorithmic_bytes_per_launch"],
+                     "launch_ms": top["ms_per_launch"],
+                     "whole_step": {"GB/s": step_gbs, "frac": step_gbs / peak, "frac_of_8000_nominal": step_gbs / 8000.0,
+                                    "algorithmic_bytes_per_step": alg_bytes, "launches_per_step": launches / args.steps},
+                     "kernels": kernels,
+                     "note": "per-kernel times from a second pass of the same steps with each launch bracketed by "
+                             "CUDA events on the launching stream; whole_step is the timed region itself"},
     }
 
     if not args.no_extras:
@@ -408,16 +466,17 @@ def main():
                      if not (r == wl.ratio and v == wl.variant)]
             for w in todo:
                 small = w.algorithmic_bytes_per_step() < 1e9
-                ms_w, launches_w, el_w, bytes_w = bench_workload(B, WL, w, w.steps, 3, None, 1, 0,
-                                                                 flush=flush if small else None)
-                gbs = bytes_w / (ms_w / max(1, launches_w) * 1e-3) / 1e9
+                ms_w, launches_w, el_w, bytes_w, _ = bench_workload(B, WL, w, w.steps, 3, None, 1, 0,
+                                                                    flush=flush if small else None)
+                gbs = bytes_w * w.steps / (ms_w * 1e-3) / 1e9
                 per.append({"cfg": w.cfg, "name": w.name, "ratio": w.ratio, "variant": WL.VARIANT_NAMES[w.variant],
                             "steps": w.steps, "ms_per_step": ms_w / w.steps, "elements_per_s": el_w * w.steps / (ms_w * 1e-3),
                             "GB/s": gbs, "frac_of_measured_peak": gbs / peak, "frac_of_8000_nominal": gbs / 8000.0,
+                            "launches_per_step": launches_w / w.steps,
                             "l2": "flushed between steps" if small else "inputs larger than L2"})
             del flush
             line["per_config"] = per
-            line["per_config_note"] = ("EF, DEF and DEF-A run the same kernel given the gradients: the variant changes only "
+            line["per_config_note"] = ("EF, DEF and DEF-A run the same kernels given the gradients: the variant changes only "
                                        "where the caller evaluates them and the returned model")
             v, sec, n = oracle_sample_run(WL, wl, 3, 1, budget_s=20.0)
             line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle",

@@ -147,6 +147,19 @@ int def_block_start(const def_ctx *ctx, uint64_t step, uint64_t seed, int64_t *s
 int def_block_start_device(const uint64_t *seeds, const uint64_t *steps, const int64_t *ds,
                            int64_t n, int64_t *starts_out, void *cuda_stream);
 
+/*
+ * Profiling aid.  A step on 16-byte aligned rows is two kernels: DEF_KERNEL_BLOCK does the
+ * tiles of 1024 coordinates that touch the block (cross-worker sum, update of params),
+ * DEF_KERNEL_STREAM all the others; narrower alignments and the d % 4 tail run
+ * DEF_KERNEL_GENERAL.  With timing enabled every launch is bracketed by CUDA events on the
+ * context's stream and WAITED for, and its device time is added to its kernel's total:
+ * calls then block, so leave it off when measuring throughput.  def_kernel_time reads the
+ * totals accumulated since def_create.
+ */
+enum { DEF_KERNEL_STREAM = 0, DEF_KERNEL_BLOCK = 1, DEF_KERNEL_GENERAL = 2, DEF_KERNEL_KINDS = 3 };
+int def_set_kernel_timing(def_ctx *ctx, int enable);
+int def_kernel_time(const def_ctx *ctx, int kernel, double *total_ms_out, int64_t *launches_out);
+
 /* Kernels this context has launched so far (every launch of every call). */
 int def_launch_count(const def_ctx *ctx, int64_t *count_out);
 

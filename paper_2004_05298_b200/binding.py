@@ -14,6 +14,7 @@ DEF_OK = 0
 DEF_ERR_ARG, DEF_ERR_NULL, DEF_ERR_ALIGN, DEF_ERR_ALIAS = -1, -2, -3, -4
 DEF_ERR_DEVICE, DEF_ERR_CUDA, DEF_ERR_UNSUPPORTED = -5, -6, -7
 DEF_MAX_WORKERS = 64
+DEF_KERNEL_STREAM, DEF_KERNEL_BLOCK, DEF_KERNEL_GENERAL = 0, 1, 2
 
 _i64, _u64, _i32, _f32, _ptr = (ctypes.c_int64, ctypes.c_uint64, ctypes.c_int32, ctypes.c_float,
                                 ctypes.c_void_p)
@@ -31,6 +32,8 @@ SIGNATURES = {
     "def_block_start": (ctypes.c_int, [_ptr, _u64, _u64, _ptr]),
     "def_block_start_device": (ctypes.c_int, [_ptr, _ptr, _ptr, _i64, _ptr, _ptr]),
     "def_launch_count": (ctypes.c_int, [_ptr, _ptr]),
+    "def_set_kernel_timing": (ctypes.c_int, [_ptr, ctypes.c_int]),
+    "def_kernel_time": (ctypes.c_int, [_ptr, ctypes.c_int, _ptr, _ptr]),
     "def_last_error": (ctypes.c_char_p, []),
 }
 
@@ -184,3 +187,14 @@ def def_launch_count(ctx):
     out = ctypes.c_int64(0)
     _check(lib.def_launch_count(ctx.handle, ctypes.byref(out)))
     return int(out.value)
+
+
+def def_set_kernel_timing(ctx, enable):
+    _check(lib.def_set_kernel_timing(ctx.handle, 1 if enable else 0))
+
+
+def def_kernel_time(ctx, kernel):
+    """(total device milliseconds, launches) of one kernel kind since def_create."""
+    ms, n = ctypes.c_double(0.0), ctypes.c_int64(0)
+    _check(lib.def_kernel_time(ctx.handle, int(kernel), ctypes.byref(ms), ctypes.byref(n)))
+    return float(ms.value), int(n.value)

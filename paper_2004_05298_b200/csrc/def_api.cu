@@ -43,6 +43,11 @@ struct def_ctx {
     float lr = 0.f, momentum = 0.f, lambda = 0.3f;
     cudaStream_t stream = nullptr;
     int64_t launches = 0;
+    // per-kernel device times (profiling aid, off by default)
+    bool timing = false;
+    cudaEvent_t t_begin = nullptr, t_end = nullptr;
+    double kernel_ms[DEF_KERNEL_KINDS] = {0.0, 0.0, 0.0};
+    int64_t kernel_launches[DEF_KERNEL_KINDS] = {0, 0, 0};
     // device facts, filled by the first launching call
     bool device_checked = false;
     int device = -1;
@@ -123,8 +128,31 @@ int vector_width(int64_t ld, const float *x, const float *g, const float *e, con
 constexpr int kBlockRows = 8;
 constexpr int kPolicy = defk::kCacheDefault;
 
+// Runs `launch` (one kernel launch on `stream`), counts it, and in timing mode brackets it
+// with events and waits for it so that its device time can be added to the kernel's total.
+template <typename Launch>
+cudaError_t counted_launch(def_ctx *ctx, int kind, cudaStream_t stream, Launch launch) {
+    if (ctx->timing) {
+        cudaError_t err = cudaEventRecord(ctx->t_begin, stream);
+        if (err != cudaSuccess) return err;
+    }
+    launch();
+    cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) return err;
+    ctx->launches += 1;
+    if (ctx->timing) {
+        float ms = 0.f;
+        if ((err = cudaEventRecord(ctx->t_end, stream)) != cudaSuccess) return err;
+        if ((err = cudaEventSynchronize(ctx->t_end)) != cudaSuccess) return err;
+        if ((err = cudaEventElapsedTime(&ms, ctx->t_begin, ctx->t_end)) != cudaSuccess) return err;
+        ctx->kernel_ms[kind] += ms;
+        ctx->kernel_launches[kind] += 1;
+    }
+    return cudaSuccess;
+}
+
 template <int V, bool MOM>
-cudaError_t launch_one(const defk::StepArgs &a, cudaStream_t stream, int64_t *launches) {
+cudaError_t launch_one(def_ctx *ctx, const defk::StepArgs &a, cudaStream_t stream) {
     const int64_t groups = a.n / V;
     if (groups == 0) return cudaSuccess;
     if (V == 4) {
@@ -132,28 +160,29 @@ cudaError_t launch_one(const defk::StepArgs &a, cudaStream_t stream, int64_t *la
         if (tiles > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
         // the few tiles that touch the block first, then the stream over all the others
         const int64_t block_ctas = a.k / defk::kTile + 4;
-        defk::def_step_block_kernel<MOM, kBlockRows, kPolicy>
-            <<<(unsigned)(block_ctas < tiles + 1 ? block_ctas : tiles + 1), defk::kTileThreads, 0, stream>>>(a);
-        cudaError_t err = cudaGetLastError();
+        const unsigned block_grid = (unsigned)(block_ctas < tiles + 1 ? block_ctas : tiles + 1);
+        cudaError_t err = counted_launch(ctx, DEF_KERNEL_BLOCK, stream, [&] {
+            defk::def_step_block_kernel<MOM, kBlockRows, kPolicy><<<block_grid, defk::kTileThreads, 0, stream>>>(a);
+        });
         if (err != cudaSuccess) return err;
-        *launches += 1;
         const dim3 grid((unsigned)tiles, (unsigned)a.W);
-        defk::def_step_stream_kernel<MOM, kPolicy><<<grid, defk::kTileThreads, 0, stream>>>(a);
-    } else {
-        // One group of V coordinates per thread; the grid-stride loop only covers the case
-        // of more groups than one grid can hold.
-        const int64_t want = (groups + kThreads - 1) / kThreads;
-        const int64_t cap = 0x7fffffffLL;
-        defk::def_step_kernel<V, MOM, 4><<<(unsigned)(want < cap ? want : cap), kThreads, 0, stream>>>(a);
+        return counted_launch(ctx, DEF_KERNEL_STREAM, stream, [&] {
+            defk::def_step_stream_kernel<MOM, kPolicy><<<grid, defk::kTileThreads, 0, stream>>>(a);
+        });
     }
-    cudaError_t err = cudaGetLastError();
-    if (err == cudaSuccess) *launches += 1;
-    return err;
+    // One group of V coordinates per thread; the grid-stride loop only covers the case of
+    // more groups than one grid can hold.
+    const int64_t want = (groups + kThreads - 1) / kThreads;
+    const int64_t cap = 0x7fffffffLL;
+    const unsigned grid = (unsigned)(want < cap ? want : cap);
+    return counted_launch(ctx, DEF_KERNEL_GENERAL, stream, [&] {
+        defk::def_step_kernel<V, MOM, 4><<<grid, kThreads, 0, stream>>>(a);
+    });
 }
 
 template <int V>
-cudaError_t launch_v(const defk::StepArgs &a, cudaStream_t stream, int64_t *launches) {
-    return a.m ? launch_one<V, true>(a, stream, launches) : launch_one<V, false>(a, stream, launches);
+cudaError_t launch_v(def_ctx *ctx, const defk::StepArgs &a, cudaStream_t stream) {
+    return a.m ? launch_one<V, true>(ctx, a, stream) : launch_one<V, false>(ctx, a, stream);
 }
 
 // Enqueue the step on local coordinates [0, n) of a view; counts launches.
@@ -170,15 +199,15 @@ int enqueue_columns(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, float *x, c
     const int64_t body = n - n % V;
     if (body > 0) {
         a.n = body;
-        err = V == 4 ? launch_v<4>(a, stream, &ctx->launches) : V == 2 ? launch_v<2>(a, stream, &ctx->launches)
-                                                              : launch_v<1>(a, stream, &ctx->launches);
+        err = V == 4 ? launch_v<4>(ctx, a, stream) : V == 2 ? launch_v<2>(ctx, a, stream)
+                                                              : launch_v<1>(ctx, a, stream);
         if (err != cudaSuccess) return cuda_fail(err, "def_step kernel launch");
     }
     if (body < n) {  // the last n % V coordinates, one float at a time
         defk::StepArgs t = a;
         t.x = x + body; t.g = g + body; t.e = e + body; t.m = m ? m + body : nullptr;
         t.n = n - body; t.j0 = j0 + body;
-        err = launch_v<1>(t, stream, &ctx->launches);
+        err = launch_v<1>(ctx, t, stream);
         if (err != cudaSuccess) return cuda_fail(err, "def_step tail kernel launch");
     }
     return DEF_OK;
@@ -290,6 +319,8 @@ def_ctx *def_create(int64_t d, int32_t W, int64_t k, int32_t variant, float lr, 
 int def_destroy(def_ctx *ctx) {
     if (!ctx) return fail(DEF_ERR_NULL, "ctx is NULL");
     free_host_path(ctx);
+    if (ctx->t_begin) cudaEventDestroy(ctx->t_begin);
+    if (ctx->t_end) cudaEventDestroy(ctx->t_end);
     delete ctx;
     return DEF_OK;
 }
@@ -330,6 +361,27 @@ int def_block_start_device(const uint64_t *seeds, const uint64_t *steps, const i
 int def_launch_count(const def_ctx *ctx, int64_t *count_out) {
     if (!ctx || !count_out) return fail(DEF_ERR_NULL, "ctx and count_out must not be NULL");
     *count_out = ctx->launches;
+    return DEF_OK;
+}
+
+int def_set_kernel_timing(def_ctx *ctx, int enable) {
+    if (!ctx) return fail(DEF_ERR_NULL, "ctx is NULL");
+    if (enable && !ctx->t_begin) {
+        int rc = check_device(ctx);
+        if (rc != DEF_OK) return rc;
+        cudaError_t err = cudaEventCreate(&ctx->t_begin);
+        if (err == cudaSuccess) err = cudaEventCreate(&ctx->t_end);
+        if (err != cudaSuccess) return cuda_fail(err, "creating timing events");
+    }
+    ctx->timing = enable != 0;
+    return DEF_OK;
+}
+
+int def_kernel_time(const def_ctx *ctx, int kernel, double *total_ms_out, int64_t *launches_out) {
+    if (!ctx || !total_ms_out || !launches_out) return fail(DEF_ERR_NULL, "NULL argument");
+    if (kernel < 0 || kernel >= DEF_KERNEL_KINDS) return fail(DEF_ERR_ARG, "unknown kernel kind %d", kernel);
+    *total_ms_out = ctx->kernel_ms[kernel];
+    *launches_out = ctx->kernel_launches[kernel];
     return DEF_OK;
 }
 

@@ -18,7 +18,7 @@ VARIANT_EF = 2
 __all__ = [
     "COMPRESSOR_RBGS", "COMPRESSOR_SCALE", "VARIANT_DEF", "VARIANT_DEF_A", "VARIANT_EF",
     "Oracle", "default", "philox4x32", "block_start", "in_block", "block_mask", "compress",
-    "step", "detach", "output",
+    "step", "detach", "output", "stats",
 ]
 
 _i64 = ctypes.c_int64
@@ -75,6 +75,9 @@ class Oracle:
             f.restype = None
             f = getattr(lib, "def_oracle_output_" + sfx)
             f.argtypes = [ctypes.c_int, _i64, _i64, _ptr, _ptr, _ptr]
+            f.restype = None
+            f = getattr(lib, "def_oracle_stats_" + sfx)
+            f.argtypes = [real, _i64, _i64, _ptr, _ptr]
             f.restype = None
 
     # ---- block start ------------------------------------------------------
@@ -159,6 +162,15 @@ class Oracle:
                                                       _p(out))
         return out
 
+    def stats(self, e, lam):
+        """(mean_k |e_k|^2, |mean_k e_k|^2, mean_k |mean e - lam e_k|^2) as Python floats."""
+        sfx, _ = _real(e.dtype)
+        W, n = e.shape
+        _check(e, e.dtype, (W, n), "e")
+        out = (ctypes.c_double * 3)()
+        getattr(self.lib, "def_oracle_stats_" + sfx)(float(lam), int(W), int(n), _p(e), out)
+        return tuple(float(v) for v in out)
+
 
 _default = None
 
@@ -201,3 +213,7 @@ def detach(x, e_w, lam):
 
 def output(variant, x, e):
     return default().output(variant, x, e)
+
+
+def stats(e, lam):
+    return default().stats(e, lam)

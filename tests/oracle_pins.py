@@ -427,6 +427,36 @@ def pin_block_start(o):
         assert len(np.unique(starts)) > 60000 or d < 10 ** 6 + 1
 
 
+# ---------------------------------------------------------------------------
+# The distances of Eq. 9: an exact small case, the special cases the text names,
+# and the expansion (1/K) sum_k |e_t - l e_k|^2 = (1 - 2l)|e_t|^2 + l^2 (1/K) sum_k |e_k|^2,
+# whose minimiser l* = |e_t|^2 / ((1/K) sum_k |e_k|^2) is the paper's lambda*(t).
+# ---------------------------------------------------------------------------
+def pin_distances(o):
+    e = np.array([[2.0, 0.0, -4.0], [0.0, 2.0, 4.0]], np.float32)       # e_t = (1, 1, 0)
+    got = o.stats(e, 0.5)
+    # (1/2)(20 + 20) = 20; |e_t|^2 = 2; e_t - e_k/2 = (0,1,2), (1,0,-2): (5 + 5)/2 = 5
+    assert got == (20.0, 2.0, 5.0), got
+    rng = _rng(47)
+    for W, n in [(1, 50), (4, 33), (7, 200)]:
+        e = rng.standard_normal((W, n)).astype(np.float32)
+        a, b, _ = o.stats(e, 0.3)
+        assert b <= a * (1 + 1e-12)                                     # |mean|^2 <= mean of squares
+        assert abs(o.stats(e, 0.0)[2] - b) <= 1e-12 * a                 # lambda = 0 is plain EF
+        if W == 1:
+            assert abs(a - b) <= 1e-12 * a and o.stats(e, 1.0)[2] <= 1e-20 * a   # K = 1, lambda = 1 vanishes
+        for lam in (0.1, 0.3, 0.8, 1.0):
+            c = o.stats(e, lam)[2]
+            lam = float(np.float32(lam))                                # the fp32 entry point takes lambda as a float
+            assert abs(c - ((1 - 2 * lam) * b + lam * lam * a)) <= 1e-12 * a, (W, n, lam)
+        best = b / a                                                    # lambda*(t)
+        if best <= 1.0:
+            at = o.stats(e, best)[2]
+            assert at <= o.stats(e, best * 0.9)[2] and at <= o.stats(e, min(1.0, best * 1.1))[2]
+        e64 = e.astype(np.float64)
+        assert np.allclose(o.stats(e64, 0.25), o.stats(e, 0.25), rtol=1e-12)
+
+
 ALL_PINS = [
     ("hand_example", pin_hand_example),
     ("telescoping_identity", pin_telescoping_identity),
@@ -443,4 +473,5 @@ ALL_PINS = [
     ("column_view", pin_column_view),
     ("philox_against_library_engine", pin_philox_against_library_engine),
     ("block_start", pin_block_start),
+    ("distances", pin_distances),
 ]

@@ -42,6 +42,11 @@ MUTANTS = [
     ("output_not_averaged", "def_oracle_body.inc", "out[i] = x[i] - sum / (REAL)W;", "out[i] = x[i] - sum;"),
     ("defa_returns_y", "def_oracle_body.inc", "if (variant == DEF_ORACLE_VARIANT_DEF) {",
      "if (variant != DEF_ORACLE_VARIANT_EF) {"),
+    ("stats_mean_not_divided", "def_oracle_body.inc", "e_t /= (double)W;", ""),
+    ("stats_detach_sign", "def_oracle_body.inc", "double diff = e_t - (double)lambda * e_k;", "double diff = e_t + (double)lambda * e_k;"),
+    ("stats_lambda_ignored", "def_oracle_body.inc", "double diff = e_t - (double)lambda * e_k;", "double diff = e_t - e_k;"),
+    ("stats_not_averaged", "def_oracle_body.inc", "out[0] = mean_sq / (double)W;", "out[0] = mean_sq;"),
+    ("stats_detached_not_averaged", "def_oracle_body.inc", "out[2] = detached / (double)W;", "out[2] = detached;"),
     ("philox_multipliers_swapped", "def_oracle.c",
      "MUL0 = 0xD2511F53u, MUL1 = 0xCD9E8D57u", "MUL0 = 0xCD9E8D57u, MUL1 = 0xD2511F53u"),
     ("philox_wrong_high_half", "def_oracle.c", "uint32_t n0 = hi1 ^ c1 ^ k0;", "uint32_t n0 = hi0 ^ c1 ^ k0;"),

@@ -262,6 +262,40 @@ def bench_workload(B, WL, wl, steps, warmup, dist, world, rank, sampler=None, fl
     return ms, launches, wl.W * d_global, alg_bytes, kernels
 
 
+def bench_aux(B, WL, wl, reps=5):
+    """Device time of the helpers around the step on the same workload: the detach point
+    (Algorithm 1 line 6), DEF's returned model and the distances of Eq. 9."""
+    import torch
+    dev = torch.device("cuda")
+    W, d = wl.W, wl.d
+    ctx = B.def_create(d, W, wl.k, WL.VARIANT_DEF, wl.lr, wl.momentum, (wl.lam, 0.0))
+    x = WL.initial_params(wl, dev)
+    e = WL.gradients(wl, 0, dev)                      # any finite values
+    z = torch.empty(W, d, dtype=torch.float32, device=dev)
+    y = torch.empty(d, dtype=torch.float32, device=dev)
+    st = torch.zeros(3, dtype=torch.float64, device=dev)
+    ops = [("def_detach", lambda: B.def_detach(ctx, x, e, z), 8 * W * d + 4 * d),
+           ("def_output", lambda: B.def_output(ctx, x, e, y), 4 * W * d + 8 * d),
+           ("def_stats", lambda: B.def_stats(ctx, e, st), 4 * W * d)]
+    out = []
+    for name, fn, nbytes in ops:
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / reps
+        out.append({"op": name, "ms": ms, "algorithmic_bytes": nbytes, "GB/s": nbytes / (ms * 1e-3) / 1e9})
+    B.def_destroy(ctx)
+    del x, e, z, y
+    torch.cuda.empty_cache()
+    return out
+
+
 def available_host_bytes():
     avail = None
     try:
@@ -475,6 +509,7 @@ def main():
                             "launches_per_step": launches_w / w.steps,
                             "l2": "flushed between steps" if small else "inputs larger than L2"})
             del flush
+            line["aux"] = bench_aux(B, WL, wl)
             line["per_config"] = per
             line["per_config_note"] = ("EF, DEF and DEF-A run the same kernels given the gradients: the variant changes only "
                                        "where the caller evaluates them and the returned model")

@@ -31,7 +31,7 @@
  *     them after the work it enqueued has run.
  *   - Calls that take device pointers only enqueue work on the context's stream
  *     (def_set_stream; default: the legacy default stream).  They do not synchronise
- *     and they allocate nothing.
+ *     and, unless a function says otherwise, allocate nothing.
  *   - Every function returns DEF_OK (0) or a negative DEF_ERR_* code and leaves a
  *     human-readable message for def_last_error() (thread-local).  Nothing is
  *     launched when validation fails.  No exception crosses this boundary.
@@ -125,6 +125,42 @@ int def_step_host(def_ctx *ctx, float *params_host, const float *grads_host, flo
 int def_step_columns_host(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, float *params_host,
                           const float *grads_host, float *errors_host, float *mom_host,
                           uint64_t step, uint64_t seed);
+
+/*
+ * The point worker w evaluates its next gradient at (Algorithm 1 line 6):
+ *     detached_out[w, j] = params[j] - lambda * errors[w, j]      (one fused multiply-add)
+ * lambda is coeffs[0] of def_create (0 for DEF_VARIANT_EF, which makes every row a copy of
+ * params).  View arguments as in def_step_columns: n coordinates, [W, n] tensors with row
+ * stride ld; the whole model is n = ld = d.  detached_out [W, ld] must not overlap the
+ * inputs (DEF_ERR_ALIAS).  Enqueued on the context's stream.
+ */
+int def_detach(def_ctx *ctx, int64_t n, int64_t ld, const float *params, const float *errors,
+               float *detached_out);
+
+/*
+ * The model Algorithm 1 returns after training (its output line):
+ *     DEF_VARIANT_DEF:            model_out[j] = params[j] - (sum_w errors[w, j]) / W
+ *                                 (y_T; workers added in order w = 0..W-1 in fp32, IEEE division)
+ *     DEF_VARIANT_DEF_A, _EF:     model_out = params (x_T); errors may be NULL
+ * model_out [n] must not overlap the inputs.  Enqueued on the context's stream.
+ */
+int def_output(def_ctx *ctx, int64_t n, int64_t ld, const float *params, const float *errors,
+               float *model_out);
+
+/*
+ * The squared distances the paper's analysis is about (Eq. 9 and the paragraph before it),
+ * over the n coordinates of the view, accumulated in fp64 from the fp32 errors:
+ *     stats_out[0] = (1/W) sum_w |e_w|^2            bound on plain EF's distance |x_t - y_t|^2
+ *     stats_out[1] = |e_bar|^2, e_bar = mean_w e_w  that distance itself
+ *     stats_out[2] = (1/W) sum_w |e_bar - lambda e_w|^2     Eq. 9, DEF's distance
+ * stats_out[2] is formed as (1 - 2 lambda) stats_out[1] + lambda^2 stats_out[0], the same
+ * quantity with the square expanded.  All three are sums over coordinates, so the results of
+ * column shards add.  stats_out: 3 doubles in DEVICE memory, written on the context's stream.
+ * Two kernels: per-CTA partial sums into a 32 KB scratch buffer the context owns (the first
+ * call allocates it with cudaMalloc; def_destroy frees it), then one CTA adds them in a fixed
+ * order, so repeated calls give identical bits.
+ */
+int def_stats(def_ctx *ctx, int64_t n, int64_t ld, const float *errors, double *stats_out);
 
 /* The stream device-pointer calls enqueue on (a cudaStream_t; NULL = legacy default). */
 int def_set_stream(def_ctx *ctx, void *cuda_stream);

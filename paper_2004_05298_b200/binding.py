@@ -27,6 +27,9 @@ SIGNATURES = {
     "def_step_columns": (ctypes.c_int, [_ptr, _i64, _i64, _i64, _ptr, _ptr, _ptr, _ptr, _u64, _u64]),
     "def_step_host": (ctypes.c_int, [_ptr, _ptr, _ptr, _ptr, _ptr, _u64, _u64]),
     "def_step_columns_host": (ctypes.c_int, [_ptr, _i64, _i64, _i64, _ptr, _ptr, _ptr, _ptr, _u64, _u64]),
+    "def_detach": (ctypes.c_int, [_ptr, _i64, _i64, _ptr, _ptr, _ptr]),
+    "def_output": (ctypes.c_int, [_ptr, _i64, _i64, _ptr, _ptr, _ptr]),
+    "def_stats": (ctypes.c_int, [_ptr, _i64, _i64, _ptr, _ptr]),
     "def_set_stream": (ctypes.c_int, [_ptr, _ptr]),
     "def_set_lr": (ctypes.c_int, [_ptr, _f32]),
     "def_block_start": (ctypes.c_int, [_ptr, _u64, _u64, _ptr]),
@@ -198,3 +201,27 @@ def def_kernel_time(ctx, kernel):
     ms, n = ctypes.c_double(0.0), ctypes.c_int64(0)
     _check(lib.def_kernel_time(ctx.handle, int(kernel), ctypes.byref(ms), ctypes.byref(n)))
     return float(ms.value), int(n.value)
+
+
+def def_detach(ctx, params, errors, detached_out, n=None, ld=None):
+    """detached_out[w] = params - lambda * errors[w]; whole model unless n / ld name a column view."""
+    n = ctx.d if n is None else int(n)
+    ld = n if ld is None else int(ld)
+    _check(lib.def_detach(ctx.handle, n, ld, _dev(params, "params", (n,)), _dev(errors, "errors", (ctx.W, ld)),
+                          _dev(detached_out, "detached_out", (ctx.W, ld))))
+
+
+def def_output(ctx, params, errors, model_out, n=None, ld=None):
+    """The model Algorithm 1 returns: y_T for DEF, x_T for DEF-A and EF."""
+    n = ctx.d if n is None else int(n)
+    ld = n if ld is None else int(ld)
+    _check(lib.def_output(ctx.handle, n, ld, _dev(params, "params", (n,)),
+                          _dev(errors, "errors", (ctx.W, ld), optional=True), _dev(model_out, "model_out", (n,))))
+
+
+def def_stats(ctx, errors, stats_out, n=None, ld=None):
+    """stats_out: 3 float64 on the GPU (see include/def.h)."""
+    n = ctx.d if n is None else int(n)
+    ld = n if ld is None else int(ld)
+    _check(lib.def_stats(ctx.handle, n, ld, _dev(errors, "errors", (ctx.W, ld)),
+                         _dev(stats_out, "stats_out", (3,), torch.float64)))

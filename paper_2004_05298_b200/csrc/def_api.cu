@@ -2,6 +2,7 @@
 // validation, kernel selection and launch, and the host-memory streaming path.
 #include "../../include/def.h"
 #include "def_kernels.cuh"
+#include "def_aux_kernels.cuh"
 
 #include <cmath>
 #include <cstdarg>
@@ -52,6 +53,8 @@ struct def_ctx {
     bool device_checked = false;
     int device = -1;
     int sm_count = 0;
+    // def_stats: per-CTA partial sums (allocated by the first def_stats call)
+    double *stats_scratch = nullptr;
     // host-memory path
     bool host_ready = false;
     int64_t host_chunk = 0;  // coordinates per staging slot (multiple of 4)
@@ -319,6 +322,7 @@ def_ctx *def_create(int64_t d, int32_t W, int64_t k, int32_t variant, float lr, 
 int def_destroy(def_ctx *ctx) {
     if (!ctx) return fail(DEF_ERR_NULL, "ctx is NULL");
     free_host_path(ctx);
+    if (ctx->stats_scratch) cudaFree(ctx->stats_scratch);
     if (ctx->t_begin) cudaEventDestroy(ctx->t_begin);
     if (ctx->t_end) cudaEventDestroy(ctx->t_end);
     delete ctx;
@@ -382,6 +386,111 @@ int def_kernel_time(const def_ctx *ctx, int kernel, double *total_ms_out, int64_
     if (kernel < 0 || kernel >= DEF_KERNEL_KINDS) return fail(DEF_ERR_ARG, "unknown kernel kind %d", kernel);
     *total_ms_out = ctx->kernel_ms[kernel];
     *launches_out = ctx->kernel_launches[kernel];
+    return DEF_OK;
+}
+
+namespace {
+
+// Shared checks of the per-coordinate helpers: a column view of n coordinates with row stride ld.
+int check_view(const def_ctx *ctx, int64_t n, int64_t ld) {
+    if (!ctx) return fail(DEF_ERR_NULL, "ctx is NULL");
+    if (n < 0 || n > ctx->d) return fail(DEF_ERR_ARG, "n=%lld is outside [0, d=%lld]", (long long)n, (long long)ctx->d);
+    if (ld < n) return fail(DEF_ERR_ARG, "row stride ld=%lld is smaller than n=%lld", (long long)ld, (long long)n);
+    return DEF_OK;
+}
+
+int width_of(int64_t ld, const void *a, const void *b, const void *c) {
+    const uintptr_t bits = (uintptr_t)a | (uintptr_t)b | (uintptr_t)c;
+    if ((bits & 15u) == 0 && ld % 4 == 0) return 4;
+    if ((bits & 7u) == 0 && ld % 2 == 0) return 2;
+    return 1;
+}
+
+}  // namespace
+
+int def_detach(def_ctx *ctx, int64_t n, int64_t ld, const float *params, const float *errors,
+               float *detached_out) {
+    int rc = check_view(ctx, n, ld);
+    if (rc != DEF_OK) return rc;
+    if (!params || !errors || !detached_out) return fail(DEF_ERR_NULL, "params, errors and detached_out must not be NULL");
+    if (((uintptr_t)params | (uintptr_t)errors | (uintptr_t)detached_out) & 3u) return fail(DEF_ERR_ALIGN, "a pointer is not 4-byte aligned");
+    const size_t rows_b = span_rows(ctx->W, n, ld), x_b = (size_t)n * sizeof(float);
+    if (overlaps(detached_out, rows_b, errors, rows_b) || overlaps(detached_out, rows_b, params, x_b))
+        return fail(DEF_ERR_ALIAS, "detached_out overlaps an input");
+    if ((rc = check_device(ctx)) != DEF_OK) return rc;
+    if (n == 0) return DEF_OK;
+    const int V = width_of(ld, params, errors, detached_out);
+    const int64_t tiles = (n + 256 * (int64_t)V - 1) / (256 * (int64_t)V);
+    const int64_t gy = tiles < 65535 ? tiles : 65535, gz = (tiles + gy - 1) / gy;
+    if (gz > 65535) return fail(DEF_ERR_ARG, "n too large");
+    const dim3 grid((unsigned)ctx->W, (unsigned)gy, (unsigned)gz);
+    if (V == 4) defk::def_detach_kernel<4><<<grid, 256, 0, ctx->stream>>>(params, errors, detached_out, n, ld, ctx->lambda);
+    else if (V == 2) defk::def_detach_kernel<2><<<grid, 256, 0, ctx->stream>>>(params, errors, detached_out, n, ld, ctx->lambda);
+    else defk::def_detach_kernel<1><<<grid, 256, 0, ctx->stream>>>(params, errors, detached_out, n, ld, ctx->lambda);
+    cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) return cuda_fail(err, "def_detach kernel launch");
+    ctx->launches += 1;
+    return DEF_OK;
+}
+
+int def_output(def_ctx *ctx, int64_t n, int64_t ld, const float *params, const float *errors,
+               float *model_out) {
+    int rc = check_view(ctx, n, ld);
+    if (rc != DEF_OK) return rc;
+    if (!params || !model_out) return fail(DEF_ERR_NULL, "params and model_out must not be NULL");
+    const bool averaged = ctx->variant == DEF_VARIANT_DEF;
+    if (averaged && !errors) return fail(DEF_ERR_NULL, "errors must not be NULL for DEF_VARIANT_DEF");
+    if (((uintptr_t)params | (uintptr_t)(averaged ? errors : nullptr) | (uintptr_t)model_out) & 3u)
+        return fail(DEF_ERR_ALIGN, "a pointer is not 4-byte aligned");
+    const size_t x_b = (size_t)n * sizeof(float);
+    if (overlaps(model_out, x_b, params, x_b) || (averaged && overlaps(model_out, x_b, errors, span_rows(ctx->W, n, ld))))
+        return fail(DEF_ERR_ALIAS, "model_out overlaps an input");
+    if ((rc = check_device(ctx)) != DEF_OK) return rc;
+    if (n == 0) return DEF_OK;
+    if (!averaged) {   // DEF-A and EF return x_T itself
+        cudaError_t err = cudaMemcpyAsync(model_out, params, x_b, cudaMemcpyDeviceToDevice, ctx->stream);
+        if (err != cudaSuccess) return cuda_fail(err, "def_output copy");
+        return DEF_OK;
+    }
+    const int V = width_of(ld, params, errors, model_out);
+    const int64_t groups = (n + V - 1) / V;
+    const int64_t blocks = (groups + 255) / 256;
+    if (blocks > 0x7fffffffLL) return fail(DEF_ERR_ARG, "n too large");
+    const float Wf = (float)ctx->W;
+    if (V == 4) defk::def_output_kernel<4, 8><<<(unsigned)blocks, 256, 0, ctx->stream>>>(params, errors, model_out, n, ld, ctx->W, Wf);
+    else if (V == 2) defk::def_output_kernel<2, 8><<<(unsigned)blocks, 256, 0, ctx->stream>>>(params, errors, model_out, n, ld, ctx->W, Wf);
+    else defk::def_output_kernel<1, 8><<<(unsigned)blocks, 256, 0, ctx->stream>>>(params, errors, model_out, n, ld, ctx->W, Wf);
+    cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) return cuda_fail(err, "def_output kernel launch");
+    ctx->launches += 1;
+    return DEF_OK;
+}
+
+int def_stats(def_ctx *ctx, int64_t n, int64_t ld, const float *errors, double *stats_out) {
+    int rc = check_view(ctx, n, ld);
+    if (rc != DEF_OK) return rc;
+    if (!errors || !stats_out) return fail(DEF_ERR_NULL, "errors and stats_out must not be NULL");
+    if (((uintptr_t)errors & 3u) || ((uintptr_t)stats_out & 7u)) return fail(DEF_ERR_ALIGN, "errors must be 4-byte and stats_out 8-byte aligned");
+    if ((rc = check_device(ctx)) != DEF_OK) return rc;
+    if (!ctx->stats_scratch) {
+        cudaError_t err = cudaMalloc(&ctx->stats_scratch, sizeof(double) * 2 * defk::kStatsMaxCtas);
+        if (err != cudaSuccess) return cuda_fail(err, "allocating def_stats scratch");
+    }
+    const int V = width_of(ld, errors, nullptr, nullptr);
+    const int64_t groups = (n + V - 1) / V;
+    int64_t ctas = (groups + defk::kStatsThreads - 1) / defk::kStatsThreads;
+    if (ctas > defk::kStatsMaxCtas) ctas = defk::kStatsMaxCtas;
+    if (ctas < 1) ctas = 1;
+    double *scratch = ctx->stats_scratch;
+    if (V == 4) defk::def_stats_partial_kernel<4, 8><<<(unsigned)ctas, defk::kStatsThreads, 0, ctx->stream>>>(errors, n, ld, ctx->W, scratch);
+    else if (V == 2) defk::def_stats_partial_kernel<2, 8><<<(unsigned)ctas, defk::kStatsThreads, 0, ctx->stream>>>(errors, n, ld, ctx->W, scratch);
+    else defk::def_stats_partial_kernel<1, 8><<<(unsigned)ctas, defk::kStatsThreads, 0, ctx->stream>>>(errors, n, ld, ctx->W, scratch);
+    cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) return cuda_fail(err, "def_stats kernel launch");
+    defk::def_stats_final_kernel<<<1, defk::kStatsThreads, 0, ctx->stream>>>(scratch, (int)ctas, ctx->W, ctx->lambda, stats_out);
+    err = cudaGetLastError();
+    if (err != cudaSuccess) return cuda_fail(err, "def_stats final kernel launch");
+    ctx->launches += 2;
     return DEF_OK;
 }
 

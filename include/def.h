@@ -162,6 +162,43 @@ int def_output(def_ctx *ctx, int64_t n, int64_t ld, const float *params, const f
  */
 int def_stats(def_ctx *ctx, int64_t n, int64_t ld, const float *errors, double *stats_out);
 
+/*
+ * def_stats for callers that cannot allocate device memory.  (The paper has no counterpart
+ * to this entry point; it exists for the integration, not for the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a framework that
+ * owns all device memory through its own pool and forbids side allocations, in a real-time
+ * or pre-sized deployment whose memory budget is fixed before start-up, or on a path where
+ * the implicit device synchronisation of cudaMalloc / cudaFree is not acceptable.  def_stats
+ * takes its 32 KB of partial-sum scratch from cudaMalloc on first use; this variant keeps the
+ * same scratch in a fixed array inside the library's device image, so it never calls
+ * cudaMalloc, cudaFree or any allocating routine.  Every GPU that loads the library holds
+ * those 32 KB (2 * DEF_STATS_STATIC_SLOTS doubles) until the process exits.
+ *
+ * It computes exactly what def_stats computes, with the same kernels, and needs no def_ctx:
+ * errors [W, ld] (device, fp32), n coordinates per row, W workers (1..DEF_MAX_WORKERS),
+ * lambda in [0, 1], stats_out = 3 doubles in device memory, cuda_stream = a cudaStream_t
+ * (NULL = legacy default stream).  The work is enqueued; nothing is synchronised.
+ *
+ * Limits and rules:
+ *   - n <= DEF_STATS_STATIC_MAX_N per call; larger n returns DEF_ERR_ARG with a message
+ *     (cut the columns into ranges and add the three results -- they are sums over
+ *     coordinates -- or use def_stats).
+ *   - The first call on each device looks up the array's device address (one query of the
+ *     runtime's symbol table, with that device current) and remembers it.  Make that first
+ *     call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps whatever the last call left
+ *     there.  A call overwrites every slot it later reads, so stale contents are harmless and
+ *     nothing is cleared; but two calls whose kernels overlap on the GPU (different streams,
+ *     or different host threads on different streams) race on it and return garbage.
+ *     Serialise them: one stream, or an event between them.
+ * Errors: DEF_ERR_NULL, DEF_ERR_ALIGN, DEF_ERR_ARG, DEF_ERR_DEVICE, DEF_ERR_CUDA.
+ */
+#define DEF_STATS_STATIC_SLOTS 2048
+#define DEF_STATS_STATIC_MAX_N ((int64_t)1 << 31)
+int def_stats_static(const float *errors, int64_t n, int64_t ld, int32_t W, float lambda,
+                     double *stats_out, void *cuda_stream);
+
 /* The stream device-pointer calls enqueue on (a cudaStream_t; NULL = legacy default). */
 int def_set_stream(def_ctx *ctx, void *cuda_stream);
 

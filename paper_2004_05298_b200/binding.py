@@ -30,6 +30,7 @@ SIGNATURES = {
     "def_detach": (ctypes.c_int, [_ptr, _i64, _i64, _ptr, _ptr, _ptr]),
     "def_output": (ctypes.c_int, [_ptr, _i64, _i64, _ptr, _ptr, _ptr]),
     "def_stats": (ctypes.c_int, [_ptr, _i64, _i64, _ptr, _ptr]),
+    "def_stats_static": (ctypes.c_int, [_ptr, _i64, _i64, _i32, _f32, _ptr, _ptr]),
     "def_set_stream": (ctypes.c_int, [_ptr, _ptr]),
     "def_set_lr": (ctypes.c_int, [_ptr, _f32]),
     "def_block_start": (ctypes.c_int, [_ptr, _u64, _u64, _ptr]),
@@ -225,3 +226,19 @@ def def_stats(ctx, errors, stats_out, n=None, ld=None):
     ld = n if ld is None else int(ld)
     _check(lib.def_stats(ctx.handle, n, ld, _dev(errors, "errors", (ctx.W, ld)),
                          _dev(stats_out, "stats_out", (3,), torch.float64)))
+
+
+DEF_STATS_STATIC_SLOTS = 2048
+DEF_STATS_STATIC_MAX_N = 1 << 31
+
+
+def def_stats_static(errors, lam, stats_out, n=None, ld=None, stream=None):
+    """def_stats without any allocation and without a context: the scratch is a fixed array in
+    the library's device image (see include/def.h for who needs this and for its rules).
+    errors: [W, ld] float32 on the GPU; stats_out: 3 float64 on the GPU."""
+    W = errors.shape[0]
+    ld = errors.shape[1] if ld is None else int(ld)
+    n = ld if n is None else int(n)
+    raw = stream.cuda_stream if isinstance(stream, torch.cuda.Stream) else (stream or 0)
+    _check(lib.def_stats_static(_dev(errors, "errors", (W, ld)), n, ld, int(W), float(lam),
+                                _dev(stats_out, "stats_out", (3,), torch.float64), ctypes.c_void_p(raw)))

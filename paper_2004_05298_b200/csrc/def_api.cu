@@ -9,6 +9,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 namespace {
@@ -577,3 +578,82 @@ int def_step_columns_host(def_ctx *ctx, int64_t c0, int64_t cols, int64_t ld, fl
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------
+// def_stats_static: the distances of def_stats for callers that must not allocate.
+//
+// The per-CTA partial sums go to this file-scope device array instead of a buffer obtained
+// with cudaMalloc.  Every GPU that loads the library carries its 32 KB until the process
+// exits.  The name below is only a host-side stand-in in host code: the address a kernel can
+// use comes from cudaGetSymbolAddress, asked for once per device with that device current.
+// ---------------------------------------------------------------------------
+static __device__ __align__(256) double g_stats_static_scratch[2 * DEF_STATS_STATIC_SLOTS];
+
+namespace {
+
+constexpr int kMaxKnownDevices = 64;
+std::mutex g_static_mutex;
+double *g_static_scratch_ptr[kMaxKnownDevices] = {};
+
+// Device address of the static scratch on the current device (looked up on first use).
+int static_scratch_address(double **ptr_out) {
+    int dev = -1;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) {
+        cudaGetLastError();
+        return fail(DEF_ERR_DEVICE, "no usable CUDA device: %s", cudaGetErrorString(err));
+    }
+    if (dev < 0 || dev >= kMaxKnownDevices) return fail(DEF_ERR_DEVICE, "device ordinal %d is not supported", dev);
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_scratch_ptr[dev]) {
+        cudaDeviceProp prop;
+        err = cudaGetDeviceProperties(&prop, dev);
+        if (err != cudaSuccess) { cudaGetLastError(); return fail(DEF_ERR_DEVICE, "cannot query device %d: %s", dev, cudaGetErrorString(err)); }
+        if (prop.major != 10)
+            return fail(DEF_ERR_DEVICE, "device %d is compute capability %d.%d; this library is built for 10.x (sm_100a)", dev, prop.major, prop.minor);
+        void *p = nullptr;
+        err = cudaGetSymbolAddress(&p, g_stats_static_scratch);
+        if (err != cudaSuccess || !p) { cudaGetLastError(); return cuda_fail(err, "cudaGetSymbolAddress(static scratch)"); }
+        g_static_scratch_ptr[dev] = static_cast<double *>(p);
+    }
+    *ptr_out = g_static_scratch_ptr[dev];
+    return DEF_OK;
+}
+
+}  // namespace
+
+extern "C" int def_stats_static(const float *errors, int64_t n, int64_t ld, int32_t W, float lambda,
+                                double *stats_out, void *cuda_stream) {
+    if (!errors || !stats_out) return fail(DEF_ERR_NULL, "errors and stats_out must not be NULL");
+    if (((uintptr_t)errors & 3u) || ((uintptr_t)stats_out & 7u))
+        return fail(DEF_ERR_ALIGN, "errors must be 4-byte and stats_out 8-byte aligned");
+    if (W < 1 || W > DEF_MAX_WORKERS) return fail(DEF_ERR_ARG, "W must be in 1..%d (got %d)", DEF_MAX_WORKERS, W);
+    if (n < 0 || n > DEF_STATS_STATIC_MAX_N)
+        return fail(DEF_ERR_ARG, "def_stats_static handles at most %lld coordinates per call (got n=%lld); "
+                                 "split the columns and add the results, or use def_stats",
+                    (long long)DEF_STATS_STATIC_MAX_N, (long long)n);
+    if (ld < n) return fail(DEF_ERR_ARG, "row stride ld=%lld is smaller than n=%lld", (long long)ld, (long long)n);
+    if (!(lambda >= 0.f && lambda <= 1.f)) return fail(DEF_ERR_ARG, "lambda must be in [0, 1]");
+    double *scratch = nullptr;
+    int rc = static_scratch_address(&scratch);
+    if (rc != DEF_OK) return rc;
+    const int V = width_of(ld, errors, nullptr, nullptr);
+    const int64_t groups = (n + V - 1) / V;
+    int64_t ctas = (groups + defk::kStatsThreads - 1) / defk::kStatsThreads;
+    if (ctas > DEF_STATS_STATIC_SLOTS) ctas = DEF_STATS_STATIC_SLOTS;
+    if (ctas < 1) ctas = 1;
+    if ((size_t)ctas * 2 * sizeof(double) > sizeof(double) * 2 * DEF_STATS_STATIC_SLOTS)
+        return fail(DEF_ERR_ARG, "the static scratch cannot hold %lld partial sums", (long long)ctas);
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    // Every slot the second kernel reads ([0, ctas)) is written by the first in this same call,
+    // so nothing left over from an earlier call is ever read and nothing needs clearing.
+    if (V == 4) defk::def_stats_partial_kernel<4, 8><<<(unsigned)ctas, defk::kStatsThreads, 0, stream>>>(errors, n, ld, W, scratch);
+    else if (V == 2) defk::def_stats_partial_kernel<2, 8><<<(unsigned)ctas, defk::kStatsThreads, 0, stream>>>(errors, n, ld, W, scratch);
+    else defk::def_stats_partial_kernel<1, 8><<<(unsigned)ctas, defk::kStatsThreads, 0, stream>>>(errors, n, ld, W, scratch);
+    cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) return cuda_fail(err, "def_stats_static kernel launch");
+    defk::def_stats_final_kernel<<<1, defk::kStatsThreads, 0, stream>>>(scratch, (int)ctas, W, lambda, stats_out);
+    err = cudaGetLastError();
+    if (err != cudaSuccess) return cuda_fail(err, "def_stats_static final kernel launch");
+    return DEF_OK;
+}

@@ -211,7 +211,7 @@ def profile_kernels(B, ctx, shard, tensors, steps, first_step, seed, per_el, k_s
     W = ctx.W
     before = {kind: B.def_kernel_time(ctx, kind) for kind in (B.DEF_KERNEL_STREAM, B.DEF_KERNEL_BLOCK, B.DEF_KERNEL_GENERAL)}
     B.def_set_kernel_timing(ctx, True)
-    bytes_stream = bytes_block = 0
+    bytes_stream = bytes_block = bytes_general = 0
     for t in range(steps):
         if flush is not None:
             flush.add_(1.0)
@@ -220,11 +220,12 @@ def profile_kernels(B, ctx, shard, tensors, steps, first_step, seed, per_el, k_s
         cols = touched_columns(ctx.d, ctx.k, B.def_block_start(ctx, step, seed), j0, n)
         bytes_block += per_el * W * cols + 8 * k_share
         bytes_stream += per_el * W * (n - cols)
+        bytes_general += per_el * W * n + 8 * k_share
     B.def_set_kernel_timing(ctx, False)
     out = []
     for kind, name, nbytes in ((B.DEF_KERNEL_STREAM, "def_step_stream_kernel", bytes_stream),
                                (B.DEF_KERNEL_BLOCK, "def_step_block_kernel", bytes_block),
-                               (B.DEF_KERNEL_GENERAL, "def_step_kernel", 0)):
+                               (B.DEF_KERNEL_GENERAL, "def_step_kernel", bytes_general)):
         ms, cnt = B.def_kernel_time(ctx, kind)
         ms, cnt = ms - before[kind][0], cnt - before[kind][1]
         if cnt:

@@ -110,6 +110,21 @@ int def_step_columns(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, float *par
                      uint64_t seed);
 
 /*
+ * def_step / def_step_columns that also write where each worker evaluates its NEXT gradient
+ * (Algorithm 1 line 6 of iteration t + 1), fused into the same two kernels:
+ *     detached_out[w, j] = x_{t+1}[j] - lambda * e_{w,t+1}[j]      (one fused multiply-add)
+ * This is the one thing that makes DEF differ from plain EF at run time (EF, lambda = 0,
+ * evaluates at x_{t+1} itself and has no use for it).  It costs one more [W, d] write:
+ * 24 instead of 20 bytes per gradient element.  detached_out [W, ld] must overlap none of
+ * the other tensors.  Other arguments and errors as for def_step / def_step_columns.
+ */
+int def_step_detach(def_ctx *ctx, float *params, const float *grads, float *errors, float *mom,
+                    float *detached_out, uint64_t step, uint64_t seed);
+int def_step_columns_detach(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, float *params,
+                            const float *grads, float *errors, float *mom, float *detached_out,
+                            uint64_t step, uint64_t seed);
+
+/*
  * One step with every tensor in HOST memory (pinned memory is much faster; pageable
  * works).  The library streams column ranges through device staging buffers it owns
  * (allocated on the first call, sized from the free device memory, freed by
@@ -201,6 +216,15 @@ int def_stats_static(const float *errors, int64_t n, int64_t ld, int32_t W, floa
 
 /* The stream device-pointer calls enqueue on (a cudaStream_t; NULL = legacy default). */
 int def_set_stream(def_ctx *ctx, void *cuda_stream);
+
+/*
+ * Launch strategy of a step on 16-byte aligned rows.  A step that moves at least `bytes`
+ * (20 * W * n) runs as the block + stream kernel pair, which is what reaches HBM speed; a
+ * smaller one is bound by launch latency and runs as one launch of the general kernel.
+ * Default 1 GiB (the measured crossover on B200); 0 always uses the pair.  Results are
+ * bit-identical either way.
+ */
+int def_set_small_step_bytes(def_ctx *ctx, int64_t bytes);
 
 /* Learning-rate schedules: eta may change between steps. */
 int def_set_lr(def_ctx *ctx, float lr);

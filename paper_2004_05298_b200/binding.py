@@ -25,6 +25,8 @@ SIGNATURES = {
     "def_destroy": (ctypes.c_int, [_ptr]),
     "def_step": (ctypes.c_int, [_ptr, _ptr, _ptr, _ptr, _ptr, _u64, _u64]),
     "def_step_columns": (ctypes.c_int, [_ptr, _i64, _i64, _i64, _ptr, _ptr, _ptr, _ptr, _u64, _u64]),
+    "def_step_detach": (ctypes.c_int, [_ptr, _ptr, _ptr, _ptr, _ptr, _ptr, _u64, _u64]),
+    "def_step_columns_detach": (ctypes.c_int, [_ptr, _i64, _i64, _i64, _ptr, _ptr, _ptr, _ptr, _ptr, _u64, _u64]),
     "def_step_host": (ctypes.c_int, [_ptr, _ptr, _ptr, _ptr, _ptr, _u64, _u64]),
     "def_step_columns_host": (ctypes.c_int, [_ptr, _i64, _i64, _i64, _ptr, _ptr, _ptr, _ptr, _u64, _u64]),
     "def_detach": (ctypes.c_int, [_ptr, _i64, _i64, _ptr, _ptr, _ptr]),
@@ -33,6 +35,7 @@ SIGNATURES = {
     "def_stats_static": (ctypes.c_int, [_ptr, _i64, _i64, _i32, _f32, _ptr, _ptr]),
     "def_set_stream": (ctypes.c_int, [_ptr, _ptr]),
     "def_set_lr": (ctypes.c_int, [_ptr, _f32]),
+    "def_set_small_step_bytes": (ctypes.c_int, [_ptr, _i64]),
     "def_block_start": (ctypes.c_int, [_ptr, _u64, _u64, _ptr]),
     "def_block_start_device": (ctypes.c_int, [_ptr, _ptr, _ptr, _i64, _ptr, _ptr]),
     "def_launch_count": (ctypes.c_int, [_ptr, _ptr]),
@@ -242,3 +245,22 @@ def def_stats_static(errors, lam, stats_out, n=None, ld=None, stream=None):
     raw = stream.cuda_stream if isinstance(stream, torch.cuda.Stream) else (stream or 0)
     _check(lib.def_stats_static(_dev(errors, "errors", (W, ld)), n, ld, int(W), float(lam),
                                 _dev(stats_out, "stats_out", (3,), torch.float64), ctypes.c_void_p(raw)))
+
+
+def def_step_detach(ctx, params, grads, errors, mom, detached_out, step, seed):
+    d, W = ctx.d, ctx.W
+    _check(lib.def_step_detach(ctx.handle, _dev(params, "params", (d,)), _dev(grads, "grads", (W, d)),
+                               _dev(errors, "errors", (W, d)), _dev(mom, "mom", (W, d), optional=True),
+                               _dev(detached_out, "detached_out", (W, d)), int(step), int(seed)))
+
+
+def def_step_columns_detach(ctx, j0, n, ld, params, grads, errors, mom, detached_out, step, seed):
+    W = ctx.W
+    _check(lib.def_step_columns_detach(ctx.handle, int(j0), int(n), int(ld), _dev(params, "params", (n,)),
+                                       _dev(grads, "grads", (W, ld)), _dev(errors, "errors", (W, ld)),
+                                       _dev(mom, "mom", (W, ld), optional=True),
+                                       _dev(detached_out, "detached_out", (W, ld)), int(step), int(seed)))
+
+
+def def_set_small_step_bytes(ctx, nbytes):
+    _check(lib.def_set_small_step_bytes(ctx.handle, int(nbytes)))

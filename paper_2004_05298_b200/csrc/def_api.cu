@@ -45,6 +45,7 @@ struct def_ctx {
     float lr = 0.f, momentum = 0.f, lambda = 0.3f;
     cudaStream_t stream = nullptr;
     int64_t launches = 0;
+    int64_t small_step_bytes = 0;  // set by def_create (kSmallStepBytesDefault)
     // per-kernel device times (profiling aid, off by default)
     bool timing = false;
     cudaEvent_t t_begin = nullptr, t_end = nullptr;
@@ -119,9 +120,22 @@ int validate_tensors(const def_ctx *ctx, int64_t n, int64_t ld, const float *x, 
     return DEF_OK;
 }
 
+// The optional detach output of a step: 4-byte aligned, overlapping none of the step's tensors.
+int validate_detach_out(const def_ctx *ctx, int64_t n, int64_t ld, const float *z, const float *x,
+                        const float *g, const float *e, const float *m) {
+    if (!z) return fail(DEF_ERR_NULL, "detached_out must not be NULL");
+    if ((uintptr_t)z & 3u) return fail(DEF_ERR_ALIGN, "detached_out is not 4-byte aligned");
+    const size_t rows_b = span_rows(ctx->W, n, ld);
+    if (overlaps(z, rows_b, x, (size_t)n * sizeof(float)) || overlaps(z, rows_b, g, rows_b) ||
+        overlaps(z, rows_b, e, rows_b) || (m && overlaps(z, rows_b, m, rows_b)))
+        return fail(DEF_ERR_ALIAS, "detached_out overlaps another tensor");
+    return DEF_OK;
+}
+
 // Widest access every row of the view supports.
-int vector_width(int64_t ld, const float *x, const float *g, const float *e, const float *m) {
-    uintptr_t bits = (uintptr_t)x | (uintptr_t)g | (uintptr_t)e | (uintptr_t)m;
+int vector_width(int64_t ld, const float *x, const float *g, const float *e, const float *m,
+                 const float *z = nullptr) {
+    uintptr_t bits = (uintptr_t)x | (uintptr_t)g | (uintptr_t)e | (uintptr_t)m | (uintptr_t)z;
     if ((bits & 15u) == 0 && ld % 4 == 0) return 4;
     if ((bits & 7u) == 0 && ld % 2 == 0) return 2;
     return 1;
@@ -155,24 +169,45 @@ cudaError_t counted_launch(def_ctx *ctx, int kind, cudaStream_t stream, Launch l
     return cudaSuccess;
 }
 
-template <int V, bool MOM>
+// With the fused detach output the W CTAs of a tile are launched next to each other
+// (grid (W, tiles)) so that the tile's x is fetched from HBM once: measured faster than
+// re-reading x for every row.
+constexpr bool kDetachWorkerFastest = true;
+
+// Below about this many bytes of [W, n] traffic a step is bound by launch and ramp-up latency,
+// not by bandwidth, and one launch of the general kernel beats the block + stream pair
+// (measured with a flushed L2: 19.5 vs 25.6 us at 80 MB, 54.5 vs 58.4 us at 320 MB, 286.8 vs
+// 283.7 us at 1.9 GB).  def_set_small_step_bytes changes it per context.
+constexpr int64_t kSmallStepBytesDefault = (int64_t)1 << 30;
+
+template <int V, bool MOM, bool DETACH>
 cudaError_t launch_one(def_ctx *ctx, const defk::StepArgs &a, cudaStream_t stream) {
     const int64_t groups = a.n / V;
     if (groups == 0) return cudaSuccess;
-    if (V == 4) {
+    if (V == 4 && 20 * (int64_t)a.W * a.n >= ctx->small_step_bytes) {
         const int64_t tiles = (a.n + defk::kTile - 1) / defk::kTile;
         if (tiles > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
         // the few tiles that touch the block first, then the stream over all the others
         const int64_t block_ctas = a.k / defk::kTile + 4;
         const unsigned block_grid = (unsigned)(block_ctas < tiles + 1 ? block_ctas : tiles + 1);
         cudaError_t err = counted_launch(ctx, DEF_KERNEL_BLOCK, stream, [&] {
-            defk::def_step_block_kernel<MOM, kBlockRows, kPolicy><<<block_grid, defk::kTileThreads, 0, stream>>>(a);
+            defk::def_step_block_kernel<MOM, kBlockRows, kPolicy, DETACH><<<block_grid, defk::kTileThreads, 0, stream>>>(a);
         });
         if (err != cudaSuccess) return err;
-        const dim3 grid((unsigned)tiles, (unsigned)a.W);
-        return counted_launch(ctx, DEF_KERNEL_STREAM, stream, [&] {
-            defk::def_step_stream_kernel<MOM, kPolicy><<<grid, defk::kTileThreads, 0, stream>>>(a);
-        });
+        if constexpr (DETACH && kDetachWorkerFastest) {
+            const int64_t gy = tiles < 65535 ? tiles : 65535, gz = (tiles + gy - 1) / gy;
+            if (gz > 65535) return cudaErrorInvalidConfiguration;
+            const dim3 grid((unsigned)a.W, (unsigned)gy, (unsigned)gz);
+            return counted_launch(ctx, DEF_KERNEL_STREAM, stream, [&] {
+                defk::def_step_stream_kernel<MOM, kPolicy, DETACH, true><<<grid, defk::kTileThreads, 0, stream>>>(a);
+            });
+        }
+        else {
+            const dim3 grid((unsigned)tiles, (unsigned)a.W);
+            return counted_launch(ctx, DEF_KERNEL_STREAM, stream, [&] {
+                defk::def_step_stream_kernel<MOM, kPolicy, DETACH, false><<<grid, defk::kTileThreads, 0, stream>>>(a);
+            });
+        }
     }
     // One group of V coordinates per thread; the grid-stride loop only covers the case of
     // more groups than one grid can hold.
@@ -180,25 +215,27 @@ cudaError_t launch_one(def_ctx *ctx, const defk::StepArgs &a, cudaStream_t strea
     const int64_t cap = 0x7fffffffLL;
     const unsigned grid = (unsigned)(want < cap ? want : cap);
     return counted_launch(ctx, DEF_KERNEL_GENERAL, stream, [&] {
-        defk::def_step_kernel<V, MOM, 4><<<grid, kThreads, 0, stream>>>(a);
+        defk::def_step_kernel<V, MOM, 4, DETACH><<<grid, kThreads, 0, stream>>>(a);
     });
 }
 
 template <int V>
 cudaError_t launch_v(def_ctx *ctx, const defk::StepArgs &a, cudaStream_t stream) {
-    return a.m ? launch_one<V, true>(ctx, a, stream) : launch_one<V, false>(ctx, a, stream);
+    if (a.z) return a.m ? launch_one<V, true, true>(ctx, a, stream) : launch_one<V, false, true>(ctx, a, stream);
+    return a.m ? launch_one<V, true, false>(ctx, a, stream) : launch_one<V, false, false>(ctx, a, stream);
 }
 
 // Enqueue the step on local coordinates [0, n) of a view; counts launches.
 int enqueue_columns(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, float *x, const float *g,
-                    float *e, float *m, uint64_t step, uint64_t seed, cudaStream_t stream) {
+                    float *e, float *m, uint64_t step, uint64_t seed, cudaStream_t stream,
+                    float *z = nullptr) {
     if (n == 0) return DEF_OK;
     defk::StepArgs a;
-    a.x = x; a.g = g; a.e = e; a.m = m;
+    a.x = x; a.g = g; a.e = e; a.m = m; a.z = z; a.lambda = ctx->lambda;
     a.n = n; a.ld = ld; a.d = ctx->d; a.j0 = j0; a.k = ctx->k; a.W = ctx->W;
     a.eta = ctx->lr; a.mu = ctx->momentum; a.W_float = (float)ctx->W;
     a.seed = seed; a.step = step;
-    const int V = vector_width(ld, x, g, e, m);
+    const int V = vector_width(ld, x, g, e, m, z);
     cudaError_t err = cudaSuccess;
     const int64_t body = n - n % V;
     if (body > 0) {
@@ -210,6 +247,7 @@ int enqueue_columns(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, float *x, c
     if (body < n) {  // the last n % V coordinates, one float at a time
         defk::StepArgs t = a;
         t.x = x + body; t.g = g + body; t.e = e + body; t.m = m ? m + body : nullptr;
+        t.z = z ? z + body : nullptr;
         t.n = n - body; t.j0 = j0 + body;
         err = launch_v<1>(ctx, t, stream);
         if (err != cudaSuccess) return cuda_fail(err, "def_step tail kernel launch");
@@ -317,6 +355,7 @@ def_ctx *def_create(int64_t d, int32_t W, int64_t k, int32_t variant, float lr, 
     if (!ctx) { fail(DEF_ERR_ARG, "out of host memory"); return nullptr; }
     ctx->d = d; ctx->W = W; ctx->k = k; ctx->variant = variant;
     ctx->lr = lr; ctx->momentum = momentum; ctx->lambda = lambda;
+    ctx->small_step_bytes = kSmallStepBytesDefault;
     return ctx;
 }
 
@@ -366,6 +405,13 @@ int def_block_start_device(const uint64_t *seeds, const uint64_t *steps, const i
 int def_launch_count(const def_ctx *ctx, int64_t *count_out) {
     if (!ctx || !count_out) return fail(DEF_ERR_NULL, "ctx and count_out must not be NULL");
     *count_out = ctx->launches;
+    return DEF_OK;
+}
+
+int def_set_small_step_bytes(def_ctx *ctx, int64_t bytes) {
+    if (!ctx) return fail(DEF_ERR_NULL, "ctx is NULL");
+    if (bytes < 0) return fail(DEF_ERR_ARG, "bytes must be >= 0");
+    ctx->small_step_bytes = bytes;
     return DEF_OK;
 }
 
@@ -421,13 +467,12 @@ int def_detach(def_ctx *ctx, int64_t n, int64_t ld, const float *params, const f
     if ((rc = check_device(ctx)) != DEF_OK) return rc;
     if (n == 0) return DEF_OK;
     const int V = width_of(ld, params, errors, detached_out);
-    const int64_t tiles = (n + 256 * (int64_t)V - 1) / (256 * (int64_t)V);
-    const int64_t gy = tiles < 65535 ? tiles : 65535, gz = (tiles + gy - 1) / gy;
-    if (gz > 65535) return fail(DEF_ERR_ARG, "n too large");
-    const dim3 grid((unsigned)ctx->W, (unsigned)gy, (unsigned)gz);
-    if (V == 4) defk::def_detach_kernel<4><<<grid, 256, 0, ctx->stream>>>(params, errors, detached_out, n, ld, ctx->lambda);
-    else if (V == 2) defk::def_detach_kernel<2><<<grid, 256, 0, ctx->stream>>>(params, errors, detached_out, n, ld, ctx->lambda);
-    else defk::def_detach_kernel<1><<<grid, 256, 0, ctx->stream>>>(params, errors, detached_out, n, ld, ctx->lambda);
+    const int64_t groups = (n + V - 1) / V;
+    const int64_t blocks = (groups + 255) / 256;
+    if (blocks > 0x7fffffffLL) return fail(DEF_ERR_ARG, "n too large");
+    if (V == 4) defk::def_detach_kernel<4, 8><<<(unsigned)blocks, 256, 0, ctx->stream>>>(params, errors, detached_out, n, ld, ctx->W, ctx->lambda);
+    else if (V == 2) defk::def_detach_kernel<2, 8><<<(unsigned)blocks, 256, 0, ctx->stream>>>(params, errors, detached_out, n, ld, ctx->W, ctx->lambda);
+    else defk::def_detach_kernel<1, 8><<<(unsigned)blocks, 256, 0, ctx->stream>>>(params, errors, detached_out, n, ld, ctx->W, ctx->lambda);
     cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) return cuda_fail(err, "def_detach kernel launch");
     ctx->launches += 1;
@@ -513,6 +558,27 @@ int def_step(def_ctx *ctx, float *params, const float *grads, float *errors, flo
              uint64_t step, uint64_t seed) {
     if (!ctx) return fail(DEF_ERR_NULL, "ctx is NULL");
     return def_step_columns(ctx, 0, ctx->d, ctx->d, params, grads, errors, mom, step, seed);
+}
+
+int def_step_columns_detach(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, float *params,
+                            const float *grads, float *errors, float *mom, float *detached_out,
+                            uint64_t step, uint64_t seed) {
+    if (!ctx) return fail(DEF_ERR_NULL, "ctx is NULL");
+    if (j0 < 0 || n < 0 || j0 > ctx->d || n > ctx->d - j0)
+        return fail(DEF_ERR_ARG, "column range [%lld, %lld) is outside [0, %lld)", (long long)j0,
+                    (long long)(j0 + n), (long long)ctx->d);
+    if (ld < n) return fail(DEF_ERR_ARG, "row stride ld=%lld is smaller than n=%lld", (long long)ld, (long long)n);
+    int rc = validate_tensors(ctx, n, ld, params, grads, errors, mom);
+    if (rc != DEF_OK) return rc;
+    if ((rc = validate_detach_out(ctx, n, ld, detached_out, params, grads, errors, mom)) != DEF_OK) return rc;
+    if ((rc = check_device(ctx)) != DEF_OK) return rc;
+    return enqueue_columns(ctx, j0, n, ld, params, grads, errors, mom, step, seed, ctx->stream, detached_out);
+}
+
+int def_step_detach(def_ctx *ctx, float *params, const float *grads, float *errors, float *mom,
+                    float *detached_out, uint64_t step, uint64_t seed) {
+    if (!ctx) return fail(DEF_ERR_NULL, "ctx is NULL");
+    return def_step_columns_detach(ctx, 0, ctx->d, ctx->d, params, grads, errors, mom, detached_out, step, seed);
 }
 
 int def_step_host(def_ctx *ctx, float *params_host, const float *grads_host, float *errors_host,

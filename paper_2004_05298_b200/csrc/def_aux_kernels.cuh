@@ -9,28 +9,35 @@ namespace defk {
 
 // ---------------------------------------------------------------------------
 // Detach point: z[w, j] = x[j] - lambda * e[w, j], one fused multiply-add per element.
-// Grid (tiles of THREADS * V coordinates, W): CTA (t, w) does worker w's row of tile t;
-// the W CTAs of a tile are adjacent in launch order, so x is fetched from HBM once.
+// One thread per V coordinates keeps its x in registers and walks the W rows, U in flight,
+// so x is read once.
 // ---------------------------------------------------------------------------
-template <int V>
+template <int V, int U>
 __global__ void __launch_bounds__(256)
 def_detach_kernel(const float *__restrict__ x, const float *__restrict__ e, float *__restrict__ z,
-                  int64_t n, int64_t ld, float lambda) {
-    // blockIdx.x runs over workers (fastest), blockIdx.y / z over tiles
-    const int64_t tile = (int64_t)blockIdx.y + (int64_t)blockIdx.z * gridDim.y;
-    const int64_t col = (tile * blockDim.x + threadIdx.x) * V;
+                  int64_t n, int64_t ld, int W, float lambda) {
+    const int64_t col = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * V;
     if (col >= n) return;
-    const size_t at = (size_t)blockIdx.x * (size_t)ld + (size_t)col;
     if (col + V <= n) {
         const Vec<V> xv = load_vec<V, kCacheDefault>(x + col);
-        const Vec<V> ev = load_vec<V, kCacheStreaming>(e + at);
-        Vec<V> zv;
+        for (int w = 0; w < W; w += U) {
+            Vec<V> ev[U];
 #pragma unroll
-        for (int i = 0; i < V; ++i) zv.v[i] = __fmaf_rn(-lambda, ev.v[i], xv.v[i]);
-        store_vec<V, kCacheStreaming>(z + at, zv);
+            for (int u = 0; u < U; ++u)
+                if (w + u < W) ev[u] = load_vec<V, kCacheDefault>(e + (size_t)(w + u) * (size_t)ld + (size_t)col);
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                if (w + u < W) {
+                    Vec<V> zv;
+#pragma unroll
+                    for (int i = 0; i < V; ++i) zv.v[i] = __fmaf_rn(-lambda, ev[u].v[i], xv.v[i]);
+                    store_vec<V, kCacheDefault>(z + (size_t)(w + u) * (size_t)ld + (size_t)col, zv);
+                }
+        }
     } else {                                   // the n % V coordinates at the end of a row
         for (int64_t c = col; c < n; ++c)
-            z[at + (c - col)] = __fmaf_rn(-lambda, e[at + (c - col)], x[c]);
+            for (int w = 0; w < W; ++w)
+                z[(size_t)w * (size_t)ld + (size_t)c] = __fmaf_rn(-lambda, e[(size_t)w * (size_t)ld + (size_t)c], x[c]);
     }
 }
 

@@ -113,6 +113,7 @@ struct StepArgs {
     const float *g;      // [W, ld]
     float *e;            // [W, ld]
     float *m;            // [W, ld] or nullptr
+    float *z;            // [W, ld] next detach points x_{t+1} - lambda e_{t+1}, or nullptr
     int64_t n;           // local coordinates
     int64_t ld;          // row stride in floats
     int64_t d;           // model size the block is drawn over
@@ -122,6 +123,7 @@ struct StepArgs {
     float eta;           // learning rate
     float mu;            // momentum constant
     float W_float;       // (float)W, the divisor of line 9
+    float lambda;        // detach coefficient (used only when z is written)
     uint64_t seed, step; // the block start is drawn from these
 };
 
@@ -158,7 +160,10 @@ __device__ __forceinline__ void worker_row(const Vec<V> &g, const Vec<V> &m, con
 
 // All W workers of the V coordinates starting at local coordinate `col`, in worker order,
 // U rows in flight at a time; then lines 9-10 on the coordinates that are in the block.
-template <int V, bool MOM, int U, int POL>
+// With DETACH, a second walk over the rows writes the next iteration's gradient points
+// z_w = x_{t+1} - lambda e_{w,t+1} (Algorithm 1 line 6); it re-reads the e' this thread has
+// just written, which is still in cache.
+template <int V, bool MOM, int U, int POL, bool DETACH = false>
 __device__ __forceinline__ void column_group(const StepArgs &a, int64_t s, int64_t col) {
     // offset of each coordinate from the block start, mod d; in the block iff < k
     int64_t off = a.j0 + col - s;
@@ -201,12 +206,39 @@ __device__ __forceinline__ void column_group(const StepArgs &a, int64_t s, int64
             }
         }
     }
-    if (any) {                                              // x -= (sum over workers) / W
+    if (!DETACH) {
+        if (any) {                                          // x -= (sum over workers) / W
 #pragma unroll
-        for (int i = 0; i < V; ++i) {
-            if (in[i]) {
-                const float C_pt = __fdiv_rn(sent[i], a.W_float);
-                a.x[col + i] = __fsub_rn(a.x[col + i], C_pt);
+            for (int i = 0; i < V; ++i) {
+                if (in[i]) {
+                    const float C_pt = __fdiv_rn(sent[i], a.W_float);
+                    a.x[col + i] = __fsub_rn(a.x[col + i], C_pt);
+                }
+            }
+        }
+        return;
+    }
+    Vec<V> x = load_vec<V, kCacheDefault>(a.x + col);
+#pragma unroll
+    for (int i = 0; i < V; ++i) {
+        if (in[i]) {
+            x.v[i] = __fsub_rn(x.v[i], __fdiv_rn(sent[i], a.W_float));
+            a.x[col + i] = x.v[i];
+        }
+    }
+    float *zp = a.z + col;
+    for (int w = 0; w < a.W; w += U) {
+        Vec<V> e[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (w + u < a.W) e[u] = load_vec<V, kCacheDefault>(ep + (size_t)(w + u) * ld);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (w + u < a.W) {
+                Vec<V> z;
+#pragma unroll
+                for (int i = 0; i < V; ++i) z.v[i] = __fmaf_rn(-a.lambda, e[u].v[i], x.v[i]);
+                store_vec<V, POL>(zp + (size_t)(w + u) * ld, z);
             }
         }
     }
@@ -215,14 +247,14 @@ __device__ __forceinline__ void column_group(const StepArgs &a, int64_t s, int64
 // General kernel: every thread owns V coordinates and walks all W rows.  Used for rows that
 // are only 4- or 8-byte aligned (V = 1, 2) and for the n % 4 tail.  Rows must be aligned
 // for V-wide access: x, g, e, m aligned to 4V bytes and ld % V == 0.
-template <int V, bool MOM, int U>
+template <int V, bool MOM, int U, bool DETACH = false>
 __global__ void __launch_bounds__(256)
 def_step_kernel(const StepArgs a) {
     const int64_t s = cta_block_start(a);
     const int64_t groups = a.n / V;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     for (int64_t grp = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; grp < groups; grp += stride)
-        column_group<V, MOM, U, kCacheDefault>(a, s, grp * V);
+        column_group<V, MOM, U, kCacheDefault, DETACH>(a, s, grp * V);
 }
 
 // Kernels for 16-byte aligned rows.  The n local coordinates are cut into tiles of
@@ -245,23 +277,34 @@ __device__ __forceinline__ bool tile_touches_block(const StepArgs &a, int64_t s,
 // tile t: three 16-byte loads and two stores per thread, few registers, full occupancy.
 // Consecutive CTAs sweep one row after the other, so the memory system sees a handful of
 // long sequential streams.  CTAs of tiles that touch the block leave at once.
-template <bool MOM, int POL>
+// With DETACH the kernel also writes z_w = x - lambda e'_w for its row (x is unchanged outside
+// the block).  WFAST then swaps the grid to (W, tiles): the W CTAs of a tile run together and
+// share one fetch of the tile's x from HBM, at the price of W interleaved row streams.
+template <bool MOM, int POL, bool DETACH = false, bool WFAST = false>
 __global__ void __launch_bounds__(kTileThreads)
 def_step_stream_kernel(const StepArgs a) {
     const int64_t s = cta_block_start(a);
-    const int64_t tile = blockIdx.x;
+    const int64_t tile = WFAST ? (int64_t)blockIdx.y + (int64_t)blockIdx.z * gridDim.y : (int64_t)blockIdx.x;
+    const unsigned w = WFAST ? blockIdx.x : blockIdx.y;
     const int64_t col = tile * kTile + (int64_t)threadIdx.x * 4;
     if (col >= a.n || tile_touches_block(a, s, tile)) return;
-    const size_t at = (size_t)blockIdx.y * (size_t)a.ld + (size_t)col;
+    const size_t at = (size_t)w * (size_t)a.ld + (size_t)col;
     const Vec<4> g = load_vec<4, POL>(a.g + at);
     const Vec<4> e = load_vec<4, POL>(a.e + at);
-    Vec<4> m, m_new, e_new;
+    Vec<4> m, m_new, e_new, x;
     if (MOM) m = load_vec<4, POL>(a.m + at);
+    if (DETACH) x = load_vec<4, kCacheDefault>(a.x + col);
     const bool none[4] = {false, false, false, false};
     float unused[4];
     worker_row<4, MOM>(g, m, e, none, a.eta, a.mu, true, m_new, e_new, unused);
     if (MOM) store_vec<4, POL>(a.m + at, m_new);
     store_vec<4, POL>(a.e + at, e_new);
+    if (DETACH) {
+        Vec<4> z;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) z.v[i] = __fmaf_rn(-a.lambda, e_new.v[i], x.v[i]);
+        store_vec<4, POL>(a.z + at, z);
+    }
 }
 
 // Tiles that touch the block: one CTA per tile walks the W rows in order (column_group).
@@ -270,7 +313,7 @@ def_step_stream_kernel(const StepArgs a) {
 // k / TILE + 4 CTAs covers every case.  CTA i takes the i-th touched tile: first those of
 // the run that starts at s, then those of the wrapped run [0, s + k - d) that the first
 // run has not already covered.  CTAs beyond the last touched tile leave.
-template <bool MOM, int U, int POL>
+template <bool MOM, int U, int POL, bool DETACH = false>
 __global__ void __launch_bounds__(kTileThreads)
 def_step_block_kernel(const StepArgs a) {
     const int64_t s = cta_block_start(a);
@@ -293,7 +336,7 @@ def_step_block_kernel(const StepArgs a) {
         if (tile > tB1 || (tile >= tA0 && tile <= tA1)) return;  // past the end, or already done as part of run A
     }
     const int64_t col = tile * kTile + (int64_t)threadIdx.x * 4;
-    if (col < a.n) column_group<4, MOM, U, POL>(a, s, col);
+    if (col < a.n) column_group<4, MOM, U, POL, DETACH>(a, s, col);
 }
 
 }  // namespace defk

@@ -108,7 +108,7 @@ def test_block_start_device_matches_oracle(B):
 # whole-tensor parity on shapes chosen to hit every code path
 # ---------------------------------------------------------------------------
 def run_whole(B, d, W, k, steps, momentum, seed, lr=0.1, offsets=(0, 0, 0, 0), sigma=0.1,
-              variant=0, special=None):
+              variant=0, special=None, pair=True):
     dev = torch.device("cuda")
     rng = np.random.default_rng(d * 31 + W * 7 + k)
     x, cx = guarded((d,), dev, offset=offsets[0])
@@ -125,6 +125,8 @@ def run_whole(B, d, W, k, steps, momentum, seed, lr=0.1, offsets=(0, 0, 0, 0), s
     x64 = xo.astype(np.float64); e64 = eo.astype(np.float64)
     m64 = mo.astype(np.float64) if momentum else None
     ctx = B.def_create(d, W, k, variant, lr, momentum)
+    if pair:
+        B.def_set_small_step_bytes(ctx, 0)          # the block + stream kernel pair even at this size
     exact = True
     for t in steps:
         gh = (sigma * rng.standard_normal((W, d))).astype(np.float32)
@@ -170,12 +172,13 @@ SHAPES = [
 
 @pytest.mark.parametrize("d,W,k", SHAPES)
 @pytest.mark.parametrize("momentum", [0.9, 0.0])
-def test_small_shapes(B, d, W, k, momentum):
+@pytest.mark.parametrize("pair", [True, False], ids=["pair", "general"])
+def test_small_shapes(B, d, W, k, momentum, pair):
     seed = 11
     wrap = find_steps(d, k, seed, lambda s: s + k > d)          # block wraps past the end
     tail = find_steps(d, k, seed, lambda s: s >= d - 1)          # starts on the last coordinate
     steps = sorted(set([0, 1, 2, 3] + wrap + tail))
-    exact = run_whole(B, d, W, k, steps, momentum, seed)
+    exact = run_whole(B, d, W, k, steps, momentum, seed, pair=pair)
     assert exact, "expected bit-identical results (same roundings in the same order)"
 
 
@@ -333,7 +336,8 @@ def test_config5_full_size_sampled(B, ratio, variant):
 # ---------------------------------------------------------------------------
 # column ranges, host memory, streams, resume
 # ---------------------------------------------------------------------------
-def test_step_columns_equals_whole_step(B):
+@pytest.mark.parametrize("pair", [True, False], ids=["pair", "general"])
+def test_step_columns_equals_whole_step(B, pair):
     dev = torch.device("cuda")
     wl = WL.get(2).scaled(200_001, W=6)
     d, W, k = wl.d, wl.W, wl.k
@@ -341,6 +345,8 @@ def test_step_columns_equals_whole_step(B):
     cuts = [0, 4, 70_000, 70_003, 150_002, d]                     # aligned and unaligned pieces
     xs = [x[a:b].clone() for a, b in zip(cuts[:-1], cuts[1:])]
     ctx = B.def_create(d, W, k, wl.variant, wl.lr, wl.momentum)
+    if pair:
+        B.def_set_small_step_bytes(ctx, 0)
     es = [torch.zeros(W, b - a + 5, device=dev) for a, b in zip(cuts[:-1], cuts[1:])]   # ld = n + 5
     ms = [torch.zeros(W, b - a + 5, device=dev) for a, b in zip(cuts[:-1], cuts[1:])]
     for t in range(6):
@@ -405,4 +411,94 @@ def test_stream_and_resume(B):
     resumed = run(range(5, 10), state=half)               # the sampler has no state to carry
     for a, b in zip(straight, resumed):
         assert torch.equal(a, b)
+    B.def_destroy(ctx)
+
+
+# ---------------------------------------------------------------------------
+# the step with the fused detach output (Algorithm 1 line 6 of the next iteration)
+# ---------------------------------------------------------------------------
+def run_detach(B, d, W, k, steps, momentum, lam, variant=0, offsets=(0, 0, 0, 0, 0), seed=7, pair=True):
+    dev = torch.device("cuda")
+    rng = np.random.default_rng(d + 13 * W + k)
+    x, cx = guarded((d,), dev, offset=offsets[0])
+    g, cg = guarded((W, d), dev, offset=offsets[1])
+    e, ce = guarded((W, d), dev, offset=offsets[2])
+    z, cz = guarded((W, d), dev, offset=offsets[4])
+    x.copy_(torch.from_numpy((0.05 * rng.standard_normal(d)).astype(np.float32))); e.zero_(); z.fill_(-3.0)
+    m = cm = None
+    if momentum:
+        m, cm = guarded((W, d), dev, offset=offsets[3]); m.zero_()
+    xo = x.cpu().numpy().copy(); eo = np.zeros((W, d), np.float32)
+    mo = np.zeros((W, d), np.float32) if momentum else None
+    ctx = B.def_create(d, W, k, variant, 0.1, momentum, (lam, 0.0))
+    if pair:
+        B.def_set_small_step_bytes(ctx, 0)
+    lam_used = 0.0 if variant == B.DEF_VARIANT_EF else lam
+    for t in steps:
+        gh = (0.1 * rng.standard_normal((W, d))).astype(np.float32)
+        g.copy_(torch.from_numpy(gh))
+        B.def_step_detach(ctx, x, g, e, m, z, t, seed)
+        oracle.step(xo, gh, eo, mo, d=d, k=k, s=oracle.block_start(seed, t, d), eta=0.1, mu=momentum)
+        zh = z.cpu().numpy()
+        for w in range(W):
+            want = oracle.detach(xo, np.ascontiguousarray(eo[w]), lam_used)
+            assert np.array_equal(zh[w], want), "detach point of worker %d differs at step %d" % (w, t)
+    assert np.array_equal(x.cpu().numpy(), xo) and np.array_equal(e.cpu().numpy(), eo)
+    if momentum:
+        assert np.array_equal(m.cpu().numpy(), mo)
+    for chk in (cx, cg, ce, cm, cz):
+        if chk:
+            chk()
+    B.def_destroy(ctx)
+
+
+@pytest.mark.parametrize("d,W,k", [(1, 1, 1), (8, 2, 3), (1025, 5, 1024), (4099, 7, 100), (65536, 64, 777),
+                                   (300000, 13, 150000), (100003, 9, 3125), (2_000_000, 4, 62_500)])
+@pytest.mark.parametrize("momentum", [0.9, 0.0])
+@pytest.mark.parametrize("pair", [True, False], ids=["pair", "general"])
+def test_step_detach_small_shapes(B, d, W, k, momentum, pair):
+    wrap = find_steps(d, k, 7, lambda s: s + k > d)
+    run_detach(B, d, W, k, sorted(set([0, 1, 2] + wrap)), momentum, 0.3, pair=pair)
+
+
+@pytest.mark.parametrize("offsets", [(0, 0, 0, 0, 0), (0, 0, 0, 0, 1), (2, 2, 2, 2, 2), (0, 1, 2, 3, 0), (0, 0, 0, 0, 2)])
+def test_step_detach_alignment_and_variants(B, offsets):
+    for d in (4096, 4098, 4099):
+        run_detach(B, d, 5, 333, [0, 1, 4], 0.9, 0.6, offsets=offsets)
+    run_detach(B, 5000, 3, 100, [0, 1], 0.9, 0.6, variant=B.DEF_VARIANT_EF)         # lambda forced to 0: z = x
+    run_detach(B, 5000, 3, 100, [0, 1], 0.9, 1.0, variant=B.DEF_VARIANT_DEF_A)
+
+
+def test_step_detach_full_size_sampled(B):
+    """Config 5 at full size: z on sampled coordinates against the oracle, and the step's own
+    outputs identical to those of the plain step."""
+    wl = WL.get(5)
+    dev = torch.device("cuda")
+    steps = 4
+    cols = sample_columns(wl, steps)
+    cols_dev = torch.from_numpy(cols).to(dev)
+    x = WL.initial_params(wl, dev); e, m = WL.zeros_state(wl, dev)
+    z = torch.empty(wl.W, wl.d, dtype=torch.float32, device=dev)
+    xo = x[cols_dev].cpu().numpy().copy()
+    n = len(cols)
+    eo = np.zeros((wl.W, n), np.float32); mo = np.zeros((wl.W, n), np.float32)
+    ctx = B.def_create(wl.d, wl.W, wl.k, wl.variant, wl.lr, wl.momentum, (wl.lam, 0.0))
+    g = torch.empty(wl.W, wl.d, dtype=torch.float32, device=dev)
+    for t in range(steps):
+        WL.gradients(wl, t, dev, out=g)
+        B.def_step_detach(ctx, x, g, e, m, z, t, wl.rbgs_seed)
+        gh = np.ascontiguousarray(g[:, cols_dev].cpu().numpy())
+        oracle.step(xo, gh, eo, mo, d=wl.d, k=wl.k, s=oracle.block_start(wl.rbgs_seed, t, wl.d), eta=wl.lr, mu=wl.momentum, cols=cols)
+        zh = z[:, cols_dev].cpu().numpy()
+        for w in range(wl.W):
+            assert np.array_equal(zh[w], oracle.detach(xo, np.ascontiguousarray(eo[w]), wl.lam)), (t, w)
+        # whole tensor: x - lambda e' in fp64, rounded to fp32.  That rounds twice where the kernel's
+        # fused multiply-add rounds once, so a handful of elements in 2e9 may differ by one ulp.
+        ref = (x.unsqueeze(0).double() - float(np.float32(wl.lam)) * e.double()).float()
+        differ = ref != z
+        assert int(differ.sum()) <= 256, "detach output differs in many places"
+        assert float((ref - z).abs().max()) <= 2.0 ** -22 * float(x.abs().max())
+        del differ
+        del ref
+    assert np.array_equal(x[cols_dev].cpu().numpy(), xo) and np.array_equal(e[:, cols_dev].cpu().numpy(), eo)
     B.def_destroy(ctx)

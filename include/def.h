@@ -125,6 +125,28 @@ int def_step_columns_detach(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, flo
                             uint64_t step, uint64_t seed);
 
 /*
+ * The step with the WORKERS cut across GPUs (the paper's own deployment: one process per
+ * GPU, each holding some of the K workers and a replica of the model; Algorithm 1 line 9 is
+ * then a real all-reduce).  A context made with W = the number of LOCAL workers runs the step
+ * in two halves around the caller's all-reduce:
+ *   def_step_rows_local  lines 7-8 (Eq. 10) for the local rows, in place as in def_step, and
+ *                        block_sum_out[i] = sum over the local workers (in order) of C(p_w) at
+ *                        block coordinate (s + i) mod d, i = 0..k-1: the k floats that travel.
+ *                        params is not needed.
+ *   (caller)             all-reduce(sum) of block_sum_out over the ranks -- additivity of the
+ *                        compressor (Assumption 3) is what makes a plain sum valid.
+ *   def_step_rows_apply  line 10: params[(s + i) mod d] -= block_sum[i] / W_total.
+ * Every rank passes the same (step, seed) and so cuts the same block.  With one rank the
+ * result equals def_step bit for bit; with several, the order in which the all-reduce adds
+ * the ranks' partial sums is the library's, so floats agree to rounding, not bitwise.
+ * RBGS only (DEF_ERR_UNSUPPORTED under DEF_COMPRESSOR_SCALE).  Whole model (n = ld = d).
+ */
+int def_step_rows_local(def_ctx *ctx, const float *grads, float *errors, float *mom,
+                        float *block_sum_out, uint64_t step, uint64_t seed);
+int def_step_rows_apply(def_ctx *ctx, float *params, const float *block_sum, int32_t W_total,
+                        uint64_t step, uint64_t seed);
+
+/*
  * One step with every tensor in HOST memory (pinned memory is much faster; pageable
  * works).  The library streams column ranges through device staging buffers it owns
  * (allocated on the first call, sized from the free device memory, freed by
@@ -216,6 +238,17 @@ int def_stats_static(const float *errors, int64_t n, int64_t ld, int32_t W, floa
 
 /* The stream device-pointer calls enqueue on (a cudaStream_t; NULL = legacy default). */
 int def_set_stream(def_ctx *ctx, void *cuda_stream);
+
+/*
+ * The compressor C of the step.  DEF_COMPRESSOR_RBGS (default) is the random block of
+ * Section 1 with the k given to def_create.  DEF_COMPRESSOR_SCALE is C(v) = delta * v,
+ * 0 < delta < 1, the case the DEF-A paragraph uses to show that x_t becomes a geometric
+ * average of the SGD iterates y_t (Eq. 11): every coordinate is sent, e' = p - delta p, and
+ * params is updated everywhere; k, step and seed are then ignored.  `delta` is ignored for
+ * RBGS.  Applies to every later step call of this context.
+ */
+enum { DEF_COMPRESSOR_RBGS = 0, DEF_COMPRESSOR_SCALE = 1 };
+int def_set_compressor(def_ctx *ctx, int32_t compressor, float delta);
 
 /*
  * Launch strategy of a step on 16-byte aligned rows.  A step that moves at least `bytes`

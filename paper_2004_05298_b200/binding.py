@@ -15,6 +15,7 @@ DEF_ERR_ARG, DEF_ERR_NULL, DEF_ERR_ALIGN, DEF_ERR_ALIAS = -1, -2, -3, -4
 DEF_ERR_DEVICE, DEF_ERR_CUDA, DEF_ERR_UNSUPPORTED = -5, -6, -7
 DEF_MAX_WORKERS = 64
 DEF_KERNEL_STREAM, DEF_KERNEL_BLOCK, DEF_KERNEL_GENERAL = 0, 1, 2
+DEF_COMPRESSOR_RBGS, DEF_COMPRESSOR_SCALE = 0, 1
 
 _i64, _u64, _i32, _f32, _ptr = (ctypes.c_int64, ctypes.c_uint64, ctypes.c_int32, ctypes.c_float,
                                 ctypes.c_void_p)
@@ -27,6 +28,8 @@ SIGNATURES = {
     "def_step_columns": (ctypes.c_int, [_ptr, _i64, _i64, _i64, _ptr, _ptr, _ptr, _ptr, _u64, _u64]),
     "def_step_detach": (ctypes.c_int, [_ptr, _ptr, _ptr, _ptr, _ptr, _ptr, _u64, _u64]),
     "def_step_columns_detach": (ctypes.c_int, [_ptr, _i64, _i64, _i64, _ptr, _ptr, _ptr, _ptr, _ptr, _u64, _u64]),
+    "def_step_rows_local": (ctypes.c_int, [_ptr, _ptr, _ptr, _ptr, _ptr, _u64, _u64]),
+    "def_step_rows_apply": (ctypes.c_int, [_ptr, _ptr, _ptr, _i32, _u64, _u64]),
     "def_step_host": (ctypes.c_int, [_ptr, _ptr, _ptr, _ptr, _ptr, _u64, _u64]),
     "def_step_columns_host": (ctypes.c_int, [_ptr, _i64, _i64, _i64, _ptr, _ptr, _ptr, _ptr, _u64, _u64]),
     "def_detach": (ctypes.c_int, [_ptr, _i64, _i64, _ptr, _ptr, _ptr]),
@@ -36,6 +39,7 @@ SIGNATURES = {
     "def_set_stream": (ctypes.c_int, [_ptr, _ptr]),
     "def_set_lr": (ctypes.c_int, [_ptr, _f32]),
     "def_set_small_step_bytes": (ctypes.c_int, [_ptr, _i64]),
+    "def_set_compressor": (ctypes.c_int, [_ptr, _i32, _f32]),
     "def_block_start": (ctypes.c_int, [_ptr, _u64, _u64, _ptr]),
     "def_block_start_device": (ctypes.c_int, [_ptr, _ptr, _ptr, _i64, _ptr, _ptr]),
     "def_launch_count": (ctypes.c_int, [_ptr, _ptr]),
@@ -264,3 +268,28 @@ def def_step_columns_detach(ctx, j0, n, ld, params, grads, errors, mom, detached
 
 def def_set_small_step_bytes(ctx, nbytes):
     _check(lib.def_set_small_step_bytes(ctx.handle, int(nbytes)))
+
+
+def def_set_compressor(ctx, compressor, delta=0.0):
+    _check(lib.def_set_compressor(ctx.handle, int(compressor), float(delta)))
+
+
+def def_step_rows_local(ctx, grads, errors, mom, block_sum_out, step, seed):
+    d, W = ctx.d, ctx.W
+    _check(lib.def_step_rows_local(ctx.handle, _dev(grads, "grads", (W, d)), _dev(errors, "errors", (W, d)),
+                                   _dev(mom, "mom", (W, d), optional=True),
+                                   _dev(block_sum_out, "block_sum_out", (ctx.k,)), int(step), int(seed)))
+
+
+def def_step_rows_apply(ctx, params, block_sum, W_total, step, seed):
+    _check(lib.def_step_rows_apply(ctx.handle, _dev(params, "params", (ctx.d,)),
+                                   _dev(block_sum, "block_sum", (ctx.k,)), int(W_total), int(step), int(seed)))
+
+
+def def_step_rows(ctx, params, grads, errors, mom, block_sum, step, seed, group=None):
+    """One row-sharded step: local half, all-reduce of the k block sums over `group` (NCCL through
+    torch.distributed, on the current stream), apply.  W_total = local W times the group size."""
+    import torch.distributed as dist
+    def_step_rows_local(ctx, grads, errors, mom, block_sum, step, seed)
+    dist.all_reduce(block_sum, op=dist.ReduceOp.SUM, group=group)
+    def_step_rows_apply(ctx, params, block_sum, ctx.W * dist.get_world_size(group), step, seed)

@@ -46,6 +46,8 @@ struct def_ctx {
     cudaStream_t stream = nullptr;
     int64_t launches = 0;
     int64_t small_step_bytes = 0;  // set by def_create (kSmallStepBytesDefault)
+    int32_t compressor = DEF_COMPRESSOR_RBGS;
+    float delta = 0.f;             // factor of DEF_COMPRESSOR_SCALE
     // per-kernel device times (profiling aid, off by default)
     bool timing = false;
     cudaEvent_t t_begin = nullptr, t_end = nullptr;
@@ -184,6 +186,13 @@ template <int V, bool MOM, bool DETACH>
 cudaError_t launch_one(def_ctx *ctx, const defk::StepArgs &a, cudaStream_t stream) {
     const int64_t groups = a.n / V;
     if (groups == 0) return cudaSuccess;
+    if (ctx->compressor == DEF_COMPRESSOR_SCALE) {   // dense: every coordinate is sent and updated
+        const int64_t want = (groups + kThreads - 1) / kThreads;
+        if (want > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+        return counted_launch(ctx, DEF_KERNEL_GENERAL, stream, [&] {
+            defk::def_step_kernel<V, MOM, 4, DETACH, true><<<(unsigned)want, kThreads, 0, stream>>>(a);
+        });
+    }
     if (V == 4 && 20 * (int64_t)a.W * a.n >= ctx->small_step_bytes) {
         const int64_t tiles = (a.n + defk::kTile - 1) / defk::kTile;
         if (tiles > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
@@ -228,10 +237,10 @@ cudaError_t launch_v(def_ctx *ctx, const defk::StepArgs &a, cudaStream_t stream)
 // Enqueue the step on local coordinates [0, n) of a view; counts launches.
 int enqueue_columns(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, float *x, const float *g,
                     float *e, float *m, uint64_t step, uint64_t seed, cudaStream_t stream,
-                    float *z = nullptr) {
+                    float *z = nullptr, float *block_sum = nullptr) {
     if (n == 0) return DEF_OK;
     defk::StepArgs a;
-    a.x = x; a.g = g; a.e = e; a.m = m; a.z = z; a.lambda = ctx->lambda;
+    a.x = x; a.g = g; a.e = e; a.m = m; a.z = z; a.block_sum = block_sum; a.lambda = ctx->lambda; a.delta = ctx->delta;
     a.n = n; a.ld = ld; a.d = ctx->d; a.j0 = j0; a.k = ctx->k; a.W = ctx->W;
     a.eta = ctx->lr; a.mu = ctx->momentum; a.W_float = (float)ctx->W;
     a.seed = seed; a.step = step;
@@ -408,6 +417,19 @@ int def_launch_count(const def_ctx *ctx, int64_t *count_out) {
     return DEF_OK;
 }
 
+int def_set_compressor(def_ctx *ctx, int32_t compressor, float delta) {
+    if (!ctx) return fail(DEF_ERR_NULL, "ctx is NULL");
+    if (compressor == DEF_COMPRESSOR_RBGS) {
+        ctx->compressor = compressor;
+        return DEF_OK;
+    }
+    if (compressor != DEF_COMPRESSOR_SCALE) return fail(DEF_ERR_ARG, "unknown compressor %d", compressor);
+    if (!(delta > 0.f && delta < 1.f)) return fail(DEF_ERR_ARG, "delta must be in (0, 1)");
+    ctx->compressor = compressor;
+    ctx->delta = delta;
+    return DEF_OK;
+}
+
 int def_set_small_step_bytes(def_ctx *ctx, int64_t bytes) {
     if (!ctx) return fail(DEF_ERR_NULL, "ctx is NULL");
     if (bytes < 0) return fail(DEF_ERR_ARG, "bytes must be >= 0");
@@ -579,6 +601,52 @@ int def_step_detach(def_ctx *ctx, float *params, const float *grads, float *erro
                     float *detached_out, uint64_t step, uint64_t seed) {
     if (!ctx) return fail(DEF_ERR_NULL, "ctx is NULL");
     return def_step_columns_detach(ctx, 0, ctx->d, ctx->d, params, grads, errors, mom, detached_out, step, seed);
+}
+
+int def_step_rows_local(def_ctx *ctx, const float *grads, float *errors, float *mom,
+                        float *block_sum_out, uint64_t step, uint64_t seed) {
+    if (!ctx) return fail(DEF_ERR_NULL, "ctx is NULL");
+    if (ctx->compressor != DEF_COMPRESSOR_RBGS)
+        return fail(DEF_ERR_UNSUPPORTED, "row-sharded steps support the RBGS compressor only");
+    if (!block_sum_out) return fail(DEF_ERR_NULL, "block_sum_out must not be NULL");
+    if ((uintptr_t)block_sum_out & 3u) return fail(DEF_ERR_ALIGN, "block_sum_out is not 4-byte aligned");
+    // params is not touched by the local half; validate the rest as usual (block_sum_out takes
+    // the place of params in the overlap checks, with its own length k)
+    if (!grads || !errors) return fail(DEF_ERR_NULL, "grads and errors must not be NULL");
+    if (ctx->momentum != 0.f && !mom) return fail(DEF_ERR_NULL, "mom must not be NULL when momentum != 0");
+    if (ctx->momentum == 0.f && mom) return fail(DEF_ERR_ARG, "mom must be NULL when momentum == 0");
+    if (((uintptr_t)grads | (uintptr_t)errors | (uintptr_t)mom) & 3u) return fail(DEF_ERR_ALIGN, "a tensor is not 4-byte aligned");
+    const size_t rows_b = span_rows(ctx->W, ctx->d, ctx->d), bs_b = (size_t)ctx->k * sizeof(float);
+    if (overlaps(grads, rows_b, errors, rows_b) || (mom && (overlaps(mom, rows_b, errors, rows_b) || overlaps(mom, rows_b, grads, rows_b))))
+        return fail(DEF_ERR_ALIAS, "grads, errors and mom must not overlap");
+    if (overlaps(block_sum_out, bs_b, grads, rows_b) || overlaps(block_sum_out, bs_b, errors, rows_b) ||
+        (mom && overlaps(block_sum_out, bs_b, mom, rows_b)))
+        return fail(DEF_ERR_ALIAS, "block_sum_out overlaps a tensor");
+    int rc = check_device(ctx);
+    if (rc != DEF_OK) return rc;
+    // x is never dereferenced when block_sum is set; the errors pointer stands in for the alignment class
+    return enqueue_columns(ctx, 0, ctx->d, ctx->d, errors, grads, errors, mom, step, seed, ctx->stream, nullptr, block_sum_out);
+}
+
+int def_step_rows_apply(def_ctx *ctx, float *params, const float *block_sum, int32_t W_total,
+                        uint64_t step, uint64_t seed) {
+    if (!ctx) return fail(DEF_ERR_NULL, "ctx is NULL");
+    if (!params || !block_sum) return fail(DEF_ERR_NULL, "params and block_sum must not be NULL");
+    if (((uintptr_t)params | (uintptr_t)block_sum) & 3u) return fail(DEF_ERR_ALIGN, "a pointer is not 4-byte aligned");
+    if (W_total < ctx->W) return fail(DEF_ERR_ARG, "W_total=%d is smaller than this context's W=%d", W_total, ctx->W);
+    if (overlaps(params, (size_t)ctx->d * sizeof(float), block_sum, (size_t)ctx->k * sizeof(float)))
+        return fail(DEF_ERR_ALIAS, "params and block_sum overlap");
+    int rc = check_device(ctx);
+    if (rc != DEF_OK) return rc;
+    defk::StepArgs a = {};
+    a.d = ctx->d; a.k = ctx->k; a.W = W_total; a.W_float = (float)W_total; a.seed = seed; a.step = step;
+    const int64_t blocks = (ctx->k + 255) / 256;
+    if (blocks > 0x7fffffffLL) return fail(DEF_ERR_ARG, "k too large");
+    defk::def_apply_block_kernel<<<(unsigned)blocks, 256, 0, ctx->stream>>>(params, block_sum, a);
+    cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) return cuda_fail(err, "def_step_rows_apply kernel launch");
+    ctx->launches += 1;
+    return DEF_OK;
 }
 
 int def_step_host(def_ctx *ctx, float *params_host, const float *grads_host, float *errors_host,

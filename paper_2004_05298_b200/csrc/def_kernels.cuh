@@ -114,6 +114,9 @@ struct StepArgs {
     float *e;            // [W, ld]
     float *m;            // [W, ld] or nullptr
     float *z;            // [W, ld] next detach points x_{t+1} - lambda e_{t+1}, or nullptr
+    float *block_sum;    // [k] or nullptr: if set, the workers' sum of C(p) on block coordinate
+                         // (s + i) mod d goes to block_sum[i] and x is left alone (rows sharded
+                         // over GPUs: the caller all-reduces block_sum, then applies it)
     int64_t n;           // local coordinates
     int64_t ld;          // row stride in floats
     int64_t d;           // model size the block is drawn over
@@ -124,6 +127,7 @@ struct StepArgs {
     float mu;            // momentum constant
     float W_float;       // (float)W, the divisor of line 9
     float lambda;        // detach coefficient (used only when z is written)
+    float delta;         // factor of the scaling compressor C(v) = delta v (used only by it)
     uint64_t seed, step; // the block start is drawn from these
 };
 
@@ -139,10 +143,13 @@ __device__ __forceinline__ int64_t cta_block_start(const StepArgs &a) {
 
 // One worker's row for V coordinates: Eq. 10 / line 7, then line 8.
 // `sent` accumulates C(p) over the workers in call order; `first` starts the sum.
-template <int V, bool MOM>
+// SCALE selects the scaling compressor C(p) = delta p of the DEF-A paragraph (the case that
+// turns the iteration into SGD with iterate averaging, Eq. 11) instead of RBGS.
+template <int V, bool MOM, bool SCALE = false>
 __device__ __forceinline__ void worker_row(const Vec<V> &g, const Vec<V> &m, const Vec<V> &e,
                                            const bool (&in)[V], float eta, float mu, bool first,
-                                           Vec<V> &m_new, Vec<V> &e_new, float (&sent)[V]) {
+                                           Vec<V> &m_new, Vec<V> &e_new, float (&sent)[V],
+                                           float delta = 0.0f) {
 #pragma unroll
     for (int i = 0; i < V; ++i) {
         float p;
@@ -152,7 +159,7 @@ __device__ __forceinline__ void worker_row(const Vec<V> &g, const Vec<V> &m, con
         } else {
             p = __fmaf_rn(eta, g.v[i], e.v[i]);              // p = eta g + e
         }
-        const float c = in[i] ? p : 0.0f;                    // C(p)
+        const float c = SCALE ? __fmul_rn(delta, p) : (in[i] ? p : 0.0f);   // C(p)
         e_new.v[i] = __fsub_rn(p, c);                        // e' = p - C(p)
         sent[i] = first ? c : __fadd_rn(sent[i], c);         // running sum of line 9
     }
@@ -163,7 +170,7 @@ __device__ __forceinline__ void worker_row(const Vec<V> &g, const Vec<V> &m, con
 // With DETACH, a second walk over the rows writes the next iteration's gradient points
 // z_w = x_{t+1} - lambda e_{w,t+1} (Algorithm 1 line 6); it re-reads the e' this thread has
 // just written, which is still in cache.
-template <int V, bool MOM, int U, int POL, bool DETACH = false>
+template <int V, bool MOM, int U, int POL, bool DETACH = false, bool SCALE = false>
 __device__ __forceinline__ void column_group(const StepArgs &a, int64_t s, int64_t col) {
     // offset of each coordinate from the block start, mod d; in the block iff < k
     int64_t off = a.j0 + col - s;
@@ -174,7 +181,7 @@ __device__ __forceinline__ void column_group(const StepArgs &a, int64_t s, int64
     for (int i = 0; i < V; ++i) {
         int64_t o = off + i;
         if (o >= a.d) o -= a.d;
-        in[i] = o < a.k;
+        in[i] = SCALE || o < a.k;                           // the scaling compressor sends every coordinate
         any |= in[i];
     }
     float sent[V];
@@ -200,7 +207,7 @@ __device__ __forceinline__ void column_group(const StepArgs &a, int64_t s, int64
             if (w + u < a.W) {
                 const size_t row = (size_t)(w + u) * ld;
                 Vec<V> m_new, e_new;
-                worker_row<V, MOM>(g[u], m[u], e[u], in, a.eta, a.mu, w + u == 0, m_new, e_new, sent);
+                worker_row<V, MOM, SCALE>(g[u], m[u], e[u], in, a.eta, a.mu, w + u == 0, m_new, e_new, sent, a.delta);
                 if (MOM) store_vec<V, POL>(mp + row, m_new);
                 store_vec<V, POL>(ep + row, e_new);
             }
@@ -211,8 +218,14 @@ __device__ __forceinline__ void column_group(const StepArgs &a, int64_t s, int64
 #pragma unroll
             for (int i = 0; i < V; ++i) {
                 if (in[i]) {
-                    const float C_pt = __fdiv_rn(sent[i], a.W_float);
-                    a.x[col + i] = __fsub_rn(a.x[col + i], C_pt);
+                    if (a.block_sum) {                      // line 9 is finished by an all-reduce
+                        int64_t o = off + i;
+                        if (o >= a.d) o -= a.d;
+                        a.block_sum[o] = sent[i];
+                    } else {
+                        const float C_pt = __fdiv_rn(sent[i], a.W_float);
+                        a.x[col + i] = __fsub_rn(a.x[col + i], C_pt);
+                    }
                 }
             }
         }
@@ -247,14 +260,14 @@ __device__ __forceinline__ void column_group(const StepArgs &a, int64_t s, int64
 // General kernel: every thread owns V coordinates and walks all W rows.  Used for rows that
 // are only 4- or 8-byte aligned (V = 1, 2) and for the n % 4 tail.  Rows must be aligned
 // for V-wide access: x, g, e, m aligned to 4V bytes and ld % V == 0.
-template <int V, bool MOM, int U, bool DETACH = false>
+template <int V, bool MOM, int U, bool DETACH = false, bool SCALE = false>
 __global__ void __launch_bounds__(256)
 def_step_kernel(const StepArgs a) {
     const int64_t s = cta_block_start(a);
     const int64_t groups = a.n / V;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     for (int64_t grp = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; grp < groups; grp += stride)
-        column_group<V, MOM, U, kCacheDefault, DETACH>(a, s, grp * V);
+        column_group<V, MOM, U, kCacheDefault, DETACH, SCALE>(a, s, grp * V);
 }
 
 // Kernels for 16-byte aligned rows.  The n local coordinates are cut into tiles of
@@ -337,6 +350,18 @@ def_step_block_kernel(const StepArgs a) {
     }
     const int64_t col = tile * kTile + (int64_t)threadIdx.x * 4;
     if (col < a.n) column_group<4, MOM, U, POL, DETACH>(a, s, col);
+}
+
+// Second half of a row-sharded step (Algorithm 1 lines 9-10 after the all-reduce):
+// x[(s + i) mod d] -= block_sum[i] / W_total for the k block coordinates.
+__global__ void __launch_bounds__(256)
+def_apply_block_kernel(float *__restrict__ x, const float *__restrict__ block_sum, StepArgs a) {
+    const int64_t s = cta_block_start(a);
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= a.k) return;
+    int64_t j = s + i;
+    if (j >= a.d) j -= a.d;
+    x[j] = __fsub_rn(x[j], __fdiv_rn(block_sum[i], a.W_float));
 }
 
 }  // namespace defk

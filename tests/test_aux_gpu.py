@@ -130,3 +130,43 @@ def test_stats_closed_form_at_full_size(B):
         total += out.cpu().numpy()
     assert np.allclose(total, got, rtol=1e-12)
     B.def_destroy(ctx)
+
+
+@pytest.mark.parametrize("d,W,offset", [(1, 1, 0), (4099, 3, 0), (100_000, 4, 0), (100_002, 8, 2), (65_537, 16, 1)])
+@pytest.mark.parametrize("momentum", [0.9, 0.0])
+def test_scaling_compressor_step(B, d, W, offset, momentum):
+    """C(v) = delta v (the DEF-A paragraph, Eq. 11): the step and its fused detach output against
+    the oracle's scaling compressor, bit for bit."""
+    dev = torch.device("cuda")
+    delta, lam, lr = 0.25, 1.0, 0.1
+    rng = np.random.default_rng(d + W)
+    x = _offset_view(torch.from_numpy((0.05 * rng.standard_normal(d)).astype(np.float32)).cuda(), offset)
+    e = _offset_view(torch.zeros(W, d, device=dev), offset)
+    m = _offset_view(torch.zeros(W, d, device=dev), offset) if momentum else None
+    z = _offset_view(torch.zeros(W, d, device=dev), offset)
+    xo = x.cpu().numpy().copy(); eo = np.zeros((W, d), np.float32)
+    mo = np.zeros((W, d), np.float32) if momentum else None
+    ctx = B.def_create(d, W, 1, B.DEF_VARIANT_DEF_A, lr, momentum, (lam, 0.0))
+    B.def_set_compressor(ctx, B.DEF_COMPRESSOR_SCALE, delta)
+    with pytest.raises(B.DefError):
+        B.def_set_compressor(ctx, B.DEF_COMPRESSOR_SCALE, 1.0)
+    for t in range(4):
+        gh = (0.1 * rng.standard_normal((W, d))).astype(np.float32)
+        g = _offset_view(torch.from_numpy(gh).cuda(), offset)
+        if t % 2:
+            B.def_step_detach(ctx, x, g, e, m, z, t, 0)
+        else:
+            B.def_step(ctx, x, g, e, m, t, 0)
+        oracle.step(xo, gh, eo, mo, d=d, k=1, s=0, eta=lr, mu=momentum, compressor=oracle.COMPRESSOR_SCALE, delta=delta)
+        assert np.array_equal(x.cpu().numpy(), xo) and np.array_equal(e.cpu().numpy(), eo), t
+        if momentum:
+            assert np.array_equal(m.cpu().numpy(), mo)
+        if t % 2:
+            for w in range(W):
+                assert np.array_equal(z[w].cpu().numpy(), oracle.detach(xo, np.ascontiguousarray(eo[w]), lam))
+    B.def_set_compressor(ctx, B.DEF_COMPRESSOR_RBGS)                     # and back: the block again
+    gh = (0.1 * rng.standard_normal((W, d))).astype(np.float32)
+    B.def_step(ctx, x, _offset_view(torch.from_numpy(gh).cuda(), offset), e, m, 9, 2)
+    oracle.step(xo, gh, eo, mo, d=d, k=1, s=oracle.block_start(2, 9, d), eta=lr, mu=momentum)
+    assert np.array_equal(x.cpu().numpy(), xo) and np.array_equal(e.cpu().numpy(), eo)
+    B.def_destroy(ctx)

@@ -79,3 +79,49 @@ def test_shard_columns_partition():
             for (a0, a1), (b0, b1) in zip(edges[:-1], edges[1:]):
                 assert a1 == b0 and a0 <= a1
             assert all(j0 % 4 == 0 or j0 == d for j0, _ in edges)      # empty trailing shards sit at d
+
+
+# ---------------------------------------------------------------------------
+# Row sharding: workers cut across ranks, Algorithm 1 line 9 as an all-reduce (gloo, CPU).
+# Each rank gets the sum of its own workers' sparsified vectors from the oracle (a step from
+# x = 0 with eta-scaled inputs moves x by minus their mean; two workers per rank keep the
+# mean's scaling exact), the ranks all-reduce those sums, and every rank applies the average.
+# ---------------------------------------------------------------------------
+def _rows_rank_main(rank, world, port, d, k, steps, out_dir):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        W_local, lr, mu = 2, 0.1, 0.9
+        rng = np.random.default_rng(77)                               # same stream on every rank
+        x = (0.05 * rng.standard_normal(d)).astype(np.float32)
+        e = np.zeros((W_local, d), np.float32); m = np.zeros((W_local, d), np.float32)
+        for t in range(steps):
+            g_all = (0.1 * rng.standard_normal((W_local * world, d))).astype(np.float32)
+            g = np.ascontiguousarray(g_all[rank * W_local:(rank + 1) * W_local])
+            s = oracle.block_start(4, t, d)
+            moved = np.zeros(d, np.float32)
+            oracle.step(moved, g, e, m, d=d, k=k, s=s, eta=lr, mu=mu)  # moved = -(local sum) / W_local
+            local_sum = torch.from_numpy(-moved * W_local)
+            dist.all_reduce(local_sum, op=dist.ReduceOp.SUM)            # the k block values (zeros elsewhere)
+            x = x - local_sum.numpy() / np.float32(W_local * world)
+        np.savez(os.path.join(out_dir, "rows%d.npz" % rank), x=x, e=e, m=m)
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_ranks_row_sharding(tmp_path):
+    world, d, k, steps = 2, 5_003, 700, 6
+    mp.spawn(_rows_rank_main, args=(world, _free_port(), d, k, steps, str(tmp_path)), nprocs=world, join=True)
+    rng = np.random.default_rng(77)
+    x = (0.05 * rng.standard_normal(d)).astype(np.float32)
+    W = 2 * world
+    e = np.zeros((W, d), np.float32); m = np.zeros((W, d), np.float32)
+    for t in range(steps):
+        g = (0.1 * rng.standard_normal((W, d))).astype(np.float32)
+        oracle.step(x, g, e, m, d=d, k=k, s=oracle.block_start(4, t, d), eta=0.1, mu=0.9)
+    parts = [np.load(tmp_path / ("rows%d.npz" % r)) for r in range(world)]
+    assert np.array_equal(parts[0]["x"], parts[1]["x"]), "replicas diverged"
+    assert np.array_equal(np.concatenate([p["e"] for p in parts]), e)
+    assert np.array_equal(np.concatenate([p["m"] for p in parts]), m)
+    assert np.max(np.abs(parts[0]["x"] - x)) <= 1e-6 * np.max(np.abs(x))

@@ -150,15 +150,18 @@ def _max_over_ranks(dist, value):
     return float(t.item())
 
 
-def time_steps(B, ctx, shard, tensors, steps, warmup, seed, dist=None, flush=None, sample_clocks=None):
+def time_steps(B, ctx, shard, tensors, steps, warmup, seed, dist=None, flush=None, sample_clocks=None, step_fn=None):
     """Device time of `steps` steps.  Without `flush`: one event pair around the whole loop,
     launches back to back.  With `flush` (a buffer larger than the L2 that is rewritten
     between iterations): one event pair per step, summed."""
     import torch
     j0, n, ld = shard
     x, g, e, m = tensors
+    if step_fn is None:
+        def step_fn(t):
+            B.def_step_columns(ctx, j0, n, ld, x, g, e, m, t, seed)
     for t in range(warmup):
-        B.def_step_columns(ctx, j0, n, ld, x, g, e, m, t, seed)
+        step_fn(t)
     _barrier(dist)
     launches0 = B.def_launch_count(ctx)
     if sample_clocks is not None:
@@ -167,7 +170,7 @@ def time_steps(B, ctx, shard, tensors, steps, warmup, seed, dist=None, flush=Non
         start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         start.record()
         for t in range(steps):
-            B.def_step_columns(ctx, j0, n, ld, x, g, e, m, warmup + t, seed)
+            step_fn(warmup + t)
         end.record()
         torch.cuda.synchronize()
         ms = start.elapsed_time(end)
@@ -177,7 +180,7 @@ def time_steps(B, ctx, shard, tensors, steps, warmup, seed, dist=None, flush=Non
             flush.add_(1.0)
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record()
-            B.def_step_columns(ctx, j0, n, ld, x, g, e, m, warmup + t, seed)
+            step_fn(warmup + t)
             b.record()
             pairs.append((a, b))
         torch.cuda.synchronize()
@@ -235,6 +238,27 @@ def profile_kernels(B, ctx, shard, tensors, steps, first_step, seed, per_el, k_s
     return out
 
 
+def bench_rows(B, WL, wl, steps, warmup, dist, world, rank, sampler=None):
+    """Workers cut across ranks (the paper's deployment): every rank holds W rows of the full model and
+    a replica of x; one step = local half, NCCL all-reduce of the k block sums, apply."""
+    import torch
+    dev = torch.device("cuda")
+    ctx = B.def_create(wl.d, wl.W, wl.k, wl.variant, wl.lr, wl.momentum, (wl.lam, 0.0))
+    x = WL.initial_params(wl, dev)
+    e, m = WL.zeros_state(wl, dev)
+    g = WL.gradients(wl, rank, dev)
+    block = torch.zeros(wl.k, dtype=torch.float32, device=dev)
+
+    def step_fn(t):
+        B.def_step_rows(ctx, x, g, e, m, block, t, wl.rbgs_seed)
+
+    ms, launches = time_steps(B, ctx, (0, wl.d, wl.d), (x, g, e, m), steps, warmup, wl.rbgs_seed, dist, None, sampler, step_fn)
+    B.def_destroy(ctx)
+    del x, g, e, m
+    torch.cuda.empty_cache()
+    return ms, launches, world * wl.W * wl.d, 20 * wl.W * wl.d + 12 * wl.k
+
+
 def bench_workload(B, WL, wl, steps, warmup, dist, world, rank, sampler=None, flush=None, profile=False):
     """Allocate a rank's shard of the workload, run, return (ms, launches, elements per step over
     all ranks, algorithmic bytes per step on this rank, per-kernel profile or None)."""
@@ -275,7 +299,16 @@ def bench_aux(B, WL, wl, reps=5):
     z = torch.empty(W, d, dtype=torch.float32, device=dev)
     y = torch.empty(d, dtype=torch.float32, device=dev)
     st = torch.zeros(3, dtype=torch.float64, device=dev)
-    ops = [("def_detach", lambda: B.def_detach(ctx, x, e, z), 8 * W * d + 4 * d),
+    g = WL.gradients(wl, 1, dev)
+    m = torch.zeros(W, d, dtype=torch.float32, device=dev)
+    counter = [0]
+
+    def fused():
+        counter[0] += 1
+        B.def_step_detach(ctx, x, g, e, m, z, counter[0], wl.rbgs_seed)
+
+    ops = [("def_step_detach", fused, 24 * W * d + 4 * d + 8 * wl.k),
+           ("def_detach", lambda: B.def_detach(ctx, x, e, z), 8 * W * d + 4 * d),
            ("def_output", lambda: B.def_output(ctx, x, e, y), 4 * W * d + 8 * d),
            ("def_stats", lambda: B.def_stats(ctx, e, st), 4 * W * d)]
     out = []
@@ -292,7 +325,7 @@ def bench_aux(B, WL, wl, reps=5):
         ms = a.elapsed_time(b) / reps
         out.append({"op": name, "ms": ms, "algorithmic_bytes": nbytes, "GB/s": nbytes / (ms * 1e-3) / 1e9})
     B.def_destroy(ctx)
-    del x, e, z, y
+    del x, e, z, y, g, m
     torch.cuda.empty_cache()
     return out
 
@@ -441,6 +474,11 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cfg", type=int, default=5, choices=[1, 2, 3, 4, 5],
                     help="workload to time (default 5, the largest; smaller ones are for profiling)")
+    ap.add_argument("--sharding", default="columns", choices=["columns", "rows"],
+                    help="columns (default): each rank holds a column range of every tensor, no collective; "
+                         "rows: each rank holds W workers of the full model and the k block sums are all-reduced (NCCL)")
+    ap.add_argument("--aux", action="store_true",
+                    help="with --no-extras: still time the helpers (detach, output, stats, step with fused detach)")
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the other workloads, the end-to-end leg and the CPU baseline")
     args = ap.parse_args()
@@ -458,6 +496,29 @@ def main():
 
     dist, world, rank, local = _dist_setup(args.gpus)
     wl = WL.get(args.cfg)
+    if args.sharding == "rows":
+        import torch.distributed as tdist
+        if dist is None:                                   # one rank: still a real NCCL group
+            tdist.init_process_group("nccl", init_method="tcp://127.0.0.1:29581", rank=0, world_size=1,
+                                     device_id=torch.device("cuda", 0))
+        sampler = ClockSampler(local)
+        ms, launches, elements, alg_bytes = bench_rows(B, WL, wl, args.steps, args.warmup, dist, world, rank, sampler)
+        clocks = sampler.finish()
+        peak, peak_kind = _measured_peak()
+        gbs = alg_bytes * args.steps / (ms * 1e-3) / 1e9
+        cfg = workload_config(wl, world)
+        cfg["parallelism"] = "workers (rows) sharded over %d GPU(s): W = %d per GPU, NCCL all-reduce of k = %d floats per step" % (world, wl.W, wl.k)
+        cfg["d"], cfg["W"], cfg["k"] = wl.d, wl.W * world, wl.k
+        if rank == 0:
+            print(json.dumps({
+                "metric": METRIC, "value": elements * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": cfg,
+                "gpu_launches": launches, "clocks": clocks,
+                "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+                             "traffic": None, "peak_kind": "of %s" % peak_kind, "kernel": "whole step (local half + all-reduce + apply)"}}))
+        tdist.destroy_process_group()
+        return
     sampler = ClockSampler(local)
     small = wl.algorithmic_bytes_per_step() < 1e9          # fits the L2: flush it between steps
     main_flush = torch.zeros(96 * 1024 * 1024, dtype=torch.float32, device="cuda") if small else None
@@ -490,6 +551,8 @@ def main():
                              "CUDA events on the launching stream; whole_step is the timed region itself"},
     }
 
+    if args.no_extras and args.aux and world == 1:
+        line["aux"] = bench_aux(B, WL, wl)
     if not args.no_extras:
         e2e_steps = max(1, min(args.steps, 3))
         line["e2e"] = bench_e2e(B, WL, wl, e2e_steps, 1, dist, world, rank)

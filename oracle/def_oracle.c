@@ -26,7 +26,7 @@
  * The float functions come in two precisions built from the same text
  * (def_oracle_body.inc): _f32 rounds like the fp32 product (one fused
  * multiply-add per update, workers summed left to right, IEEE division by W),
- * _f64 is the high-precision shadow the fp32 results are judged against.
+ * _f64 is the high-precision shadow the fp32 results are compared with.
  *
  * Pins (tests/test_oracle_*.py): hand-worked 8-coordinate example, the
  * telescoping identity of Eq. 8 with and without momentum (Eq. 10), k = d

@@ -502,3 +502,29 @@ def test_step_detach_full_size_sampled(B):
         del ref
     assert np.array_equal(x[cols_dev].cpu().numpy(), xo) and np.array_equal(e[:, cols_dev].cpu().numpy(), eo)
     B.def_destroy(ctx)
+
+
+def test_padded_rows_keep_the_kernel_pair(B):
+    """An odd d with rows padded to a multiple of 4 floats runs the 128-bit kernels (plus a
+    one-float-wide launch for the last d % 4 coordinates) and still matches the oracle."""
+    dev = torch.device("cuda")
+    d, W, k = 300_003, 6, 20_000
+    ld = (d + 3) // 4 * 4
+    rng = np.random.default_rng(9)
+    x = torch.from_numpy((0.05 * rng.standard_normal(d)).astype(np.float32)).to(dev)
+    e = torch.zeros(W, ld, device=dev); m = torch.zeros(W, ld, device=dev)
+    xo = x.cpu().numpy().copy(); eo = np.zeros((W, d), np.float32); mo = np.zeros((W, d), np.float32)
+    ctx = B.def_create(d, W, k, 0, 0.1, 0.9)
+    B.def_set_small_step_bytes(ctx, 0)
+    B.def_set_kernel_timing(ctx, True)
+    for t in range(4):
+        gh = (0.1 * rng.standard_normal((W, d))).astype(np.float32)
+        g = torch.zeros(W, ld, device=dev); g[:, :d] = torch.from_numpy(gh).to(dev)
+        B.def_step_columns(ctx, 0, d, ld, x, g, e, m, t, 6)
+        oracle.step(xo, gh, eo, mo, d=d, k=k, s=oracle.block_start(6, t, d), eta=0.1, mu=0.9)
+    assert B.def_kernel_time(ctx, B.DEF_KERNEL_STREAM)[1] == 4 and B.def_kernel_time(ctx, B.DEF_KERNEL_BLOCK)[1] == 4
+    assert B.def_kernel_time(ctx, B.DEF_KERNEL_GENERAL)[1] == 4          # the 3-coordinate tail
+    assert np.array_equal(x.cpu().numpy(), xo)
+    assert np.array_equal(e[:, :d].cpu().numpy(), eo) and np.array_equal(m[:, :d].cpu().numpy(), mo)
+    assert not e[:, d:].any() and not m[:, d:].any()
+    B.def_destroy(ctx)

@@ -442,7 +442,7 @@ def run_reference(args):
         return
     from paper_2004_05298_b200 import workloads as WL
     wl = WL.get(5)
-    value, sec, n = oracle_sample_run(WL, wl, args.steps, args.warmup, budget_s=90.0)
+    value, sec, n = oracle_sample_run(WL, wl, args.steps, args.warmup, budget_s=args.reference_budget_s)
     sample = "each step = one oracle step on columns [0, %d) of d = %d, all W = %d workers" % (n, wl.d, wl.W)
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
@@ -477,6 +477,8 @@ def main():
     ap.add_argument("--sharding", default="columns", choices=["columns", "rows"],
                     help="columns (default): each rank holds a column range of every tensor, no collective; "
                          "rows: each rank holds W workers of the full model and the k block sums are all-reduced (NCCL)")
+    ap.add_argument("--reference-budget-s", type=float, default=90.0,
+                    help="--impl reference: CPU seconds the whole run (warm-up + steps) may take")
     ap.add_argument("--aux", action="store_true",
                     help="with --no-extras: still time the helpers (detach, output, stats, step with fused detach)")
     ap.add_argument("--no-extras", action="store_true",

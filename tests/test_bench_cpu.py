@@ -1,0 +1,47 @@
+"""Host-side pieces of bench.py that need no GPU: the split of a step's bytes between the two
+kernels, and the reference arm (the CPU oracle timed on a bounded sample), which must print
+the contract's JSON line."""
+import importlib.util
+import json
+import os
+import random
+import subprocess
+import sys
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _bench():
+    spec = importlib.util.spec_from_file_location("bench_module", os.path.join(ROOT, "bench.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    return mod
+
+
+def test_touched_columns_against_brute_force():
+    bench = _bench()
+    rnd = random.Random(1)
+    for _ in range(1500):
+        d = rnd.randint(1, 9000); k = rnd.randint(1, d); s = rnd.randrange(d)
+        j0 = rnd.randrange(d); n = rnd.randint(1, d - j0)
+        block = {(s + i) % d for i in range(k)}
+        tiles = {(j - j0) // bench.TILE for j in range(j0, j0 + n) if j in block}
+        want = sum(min(bench.TILE, n - t * bench.TILE) for t in tiles)
+        assert bench.touched_columns(d, k, s, j0, n) == want, (d, k, s, j0, n)
+
+
+def test_reference_arm_prints_the_contract_line():
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "2",
+                          "--warmup", "3", "--reference-budget-s", "3"], capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0, out.stderr
+    line = json.loads(out.stdout.strip().splitlines()[-1])
+    assert line["impl"] == "reference" and line["unit"] == "elements/s" and line["higher_is_better"] is True
+    assert line["value"] > 0 and line["steps"] == 2 and line["vs_baseline"] is None
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] == 1
+    assert line["e2e"]["value"] == line["value"] and line["e2e"]["h2d_bytes_per_step"] == 0
+    assert "cfg5" in line["config"]["workload"]
+    # other ranks of a multi-process launch do no work and print nothing
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2")
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2"],
+                         capture_output=True, text=True, timeout=120, env=env)
+    assert out.returncode == 0 and out.stdout.strip() == ""

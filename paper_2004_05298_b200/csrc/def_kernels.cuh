@@ -293,13 +293,16 @@ __device__ __forceinline__ bool tile_touches_block(const StepArgs &a, int64_t s,
 // With DETACH the kernel also writes z_w = x - lambda e'_w for its row (x is unchanged outside
 // the block).  WFAST then swaps the grid to (W, tiles): the W CTAs of a tile run together and
 // share one fetch of the tile's x from HBM, at the price of W interleaved row streams.
-template <bool MOM, int POL, bool DETACH = false, bool WFAST = false>
-__global__ void __launch_bounds__(kTileThreads)
+// TILES CTAs' worth of tiles share one CTA of TILES * kTileThreads threads (each group of
+// kTileThreads threads still owns one tile and decides for it alone).
+template <bool MOM, int POL, bool DETACH = false, bool WFAST = false, int TILES = 1>
+__global__ void __launch_bounds__(kTileThreads * TILES)
 def_step_stream_kernel(const StepArgs a) {
     const int64_t s = cta_block_start(a);
-    const int64_t tile = WFAST ? (int64_t)blockIdx.y + (int64_t)blockIdx.z * gridDim.y : (int64_t)blockIdx.x;
+    const int64_t first = WFAST ? (int64_t)blockIdx.y + (int64_t)blockIdx.z * gridDim.y : (int64_t)blockIdx.x;
+    const int64_t tile = first * TILES + (int64_t)(threadIdx.x / kTileThreads);
     const unsigned w = WFAST ? blockIdx.x : blockIdx.y;
-    const int64_t col = tile * kTile + (int64_t)threadIdx.x * 4;
+    const int64_t col = tile * kTile + (int64_t)(threadIdx.x % kTileThreads) * 4;
     if (col >= a.n || tile_touches_block(a, s, tile)) return;
     const size_t at = (size_t)w * (size_t)a.ld + (size_t)col;
     const Vec<4> g = load_vec<4, POL>(a.g + at);

@@ -105,7 +105,8 @@ int def_step(def_ctx *ctx, float *params, const float *grads, float *errors, flo
  * a model can be cut by columns across GPUs, or streamed through the GPU in pieces,
  * with no exchange between the pieces.  params points at the n local coordinates;
  * grads / errors / mom point at local [W, n] tensors with row stride ld >= n floats.
- * The block start is still drawn over the whole d.  0 <= j0, j0 + n <= d.
+ * The block start is still drawn over the whole d.  0 <= j0, j0 + n <= d; n = 0 is a no-op
+ * (pointers are then not looked at).
  */
 int def_step_columns(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, float *params,
                      const float *grads, float *errors, float *mom, uint64_t step,

@@ -575,6 +575,7 @@ int def_step_columns(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, float *par
         return fail(DEF_ERR_ARG, "column range [%lld, %lld) is outside [0, %lld)", (long long)j0,
                     (long long)(j0 + n), (long long)ctx->d);
     if (ld < n) return fail(DEF_ERR_ARG, "row stride ld=%lld is smaller than n=%lld", (long long)ld, (long long)n);
+    if (n == 0) return DEF_OK;   // an empty column range (a rank with no columns) is a no-op
     int rc = validate_tensors(ctx, n, ld, params, grads, errors, mom);
     if (rc != DEF_OK) return rc;
     if ((rc = check_device(ctx)) != DEF_OK) return rc;
@@ -595,6 +596,7 @@ int def_step_columns_detach(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, flo
         return fail(DEF_ERR_ARG, "column range [%lld, %lld) is outside [0, %lld)", (long long)j0,
                     (long long)(j0 + n), (long long)ctx->d);
     if (ld < n) return fail(DEF_ERR_ARG, "row stride ld=%lld is smaller than n=%lld", (long long)ld, (long long)n);
+    if (n == 0) return DEF_OK;   // an empty column range (a rank with no columns) is a no-op
     int rc = validate_tensors(ctx, n, ld, params, grads, errors, mom);
     if (rc != DEF_OK) return rc;
     if ((rc = validate_detach_out(ctx, n, ld, detached_out, params, grads, errors, mom)) != DEF_OK) return rc;
@@ -669,6 +671,7 @@ int def_step_columns_host(def_ctx *ctx, int64_t c0, int64_t cols, int64_t ld, fl
         return fail(DEF_ERR_ARG, "column range [%lld, %lld) is outside [0, %lld)", (long long)c0,
                     (long long)(c0 + cols), (long long)ctx->d);
     if (ld < cols) return fail(DEF_ERR_ARG, "row stride ld=%lld is smaller than n=%lld", (long long)ld, (long long)cols);
+    if (cols == 0) return DEF_OK;
     int rc = validate_tensors(ctx, cols, ld, params_host, grads_host, errors_host, mom_host);
     if (rc != DEF_OK) return rc;
     if ((rc = check_device(ctx)) != DEF_OK) return rc;

@@ -528,3 +528,14 @@ def test_padded_rows_keep_the_kernel_pair(B):
     assert np.array_equal(e[:, :d].cpu().numpy(), eo) and np.array_equal(m[:, :d].cpu().numpy(), mo)
     assert not e[:, d:].any() and not m[:, d:].any()
     B.def_destroy(ctx)
+
+
+def test_empty_ranges_are_no_ops(B):
+    dev = torch.device("cuda")
+    ctx = B.def_create(1000, 2, 10, 0, 0.1, 0.9)
+    x = torch.ones(0, device=dev); t2 = torch.ones(2, 0, device=dev)
+    before = B.def_launch_count(ctx)
+    B.def_step_columns(ctx, 500, 0, 0, x, t2, t2.clone(), t2.clone(), 0, 0)
+    B.def_step_columns(ctx, 1000, 0, 0, x, t2, t2.clone(), t2.clone(), 0, 0)
+    assert B.def_launch_count(ctx) == before
+    B.def_destroy(ctx)

@@ -172,10 +172,13 @@ cudaError_t counted_launch(def_ctx *ctx, int kind, cudaStream_t stream, Launch l
     return cudaSuccess;
 }
 
-// With the fused detach output the W CTAs of a tile are launched next to each other
-// (grid (W, tiles)) so that the tile's x is fetched from HBM once: measured faster than
-// re-reading x for every row.
-constexpr bool kDetachWorkerFastest = true;
+// With the fused detach output x becomes a stream every worker's CTA of a tile reads.  The
+// stream kernel then runs in chunked order: 256 CTAs (two tiles each: 2 MB of every row and
+// of x) sweep a segment of row 0, the next 256 the same segment of row 1, and so on, so the
+// streams stay long and sequential while the segment of x stays in the L2 for all W rows.
+// Measured on the VGG-16-sized workload: 8.12 ms, against 8.78 ms with the W CTAs of a tile
+// adjacent and 8.97 ms row after row (x re-read from HBM for every row).
+constexpr int kDetachChunkCtas = 256;
 
 // Below about this many bytes of [W, n] traffic a step is bound by launch and ramp-up latency,
 // not by bandwidth, and one launch of the general kernel beats the block + stream pair
@@ -204,21 +207,25 @@ cudaError_t launch_one(def_ctx *ctx, const defk::StepArgs &a, cudaStream_t strea
             defk::def_step_block_kernel<MOM, kBlockRows, kPolicy, DETACH><<<block_grid, defk::kTileThreads, 0, stream>>>(a);
         });
         if (err != cudaSuccess) return err;
-        if constexpr (DETACH && kDetachWorkerFastest) {
-            const int64_t gy = tiles < 65535 ? tiles : 65535, gz = (tiles + gy - 1) / gy;
-            if (gz > 65535) return cudaErrorInvalidConfiguration;
-            const dim3 grid((unsigned)a.W, (unsigned)gy, (unsigned)gz);
+        constexpr int kStreamTiles = 2;
+        const int64_t slots = (tiles + kStreamTiles - 1) / kStreamTiles;
+        if constexpr (DETACH) {
+            const int64_t segments = (slots + kDetachChunkCtas - 1) / kDetachChunkCtas;
+            const int64_t ctas = segments * kDetachChunkCtas * a.W;
+            if (ctas > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+            defk::StepArgs c = a;
+            c.chunk = kDetachChunkCtas;
             return counted_launch(ctx, DEF_KERNEL_STREAM, stream, [&] {
-                defk::def_step_stream_kernel<MOM, kPolicy, DETACH, true><<<grid, defk::kTileThreads, 0, stream>>>(a);
+                defk::def_step_stream_kernel<MOM, kPolicy, true, defk::kOrderChunked, kStreamTiles>
+                    <<<(unsigned)ctas, defk::kTileThreads * kStreamTiles, 0, stream>>>(c);
             });
         }
         else {
             // two tiles per CTA of 512 threads: 0.4-0.9 % faster than one tile per 256 (half as
             // many block-start computations), while 1024 threads lose 20 %
-            constexpr int kStreamTiles = 2;
-            const dim3 grid((unsigned)((tiles + kStreamTiles - 1) / kStreamTiles), (unsigned)a.W);
+            const dim3 grid((unsigned)slots, (unsigned)a.W);
             return counted_launch(ctx, DEF_KERNEL_STREAM, stream, [&] {
-                defk::def_step_stream_kernel<MOM, kPolicy, DETACH, false, kStreamTiles>
+                defk::def_step_stream_kernel<MOM, kPolicy, false, defk::kOrderRows, kStreamTiles>
                     <<<grid, defk::kTileThreads * kStreamTiles, 0, stream>>>(a);
             });
         }
@@ -248,7 +255,7 @@ int enqueue_columns(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, float *x, c
     a.x = x; a.g = g; a.e = e; a.m = m; a.z = z; a.block_sum = block_sum; a.lambda = ctx->lambda; a.delta = ctx->delta;
     a.n = n; a.ld = ld; a.d = ctx->d; a.j0 = j0; a.k = ctx->k; a.W = ctx->W;
     a.eta = ctx->lr; a.mu = ctx->momentum; a.W_float = (float)ctx->W;
-    a.seed = seed; a.step = step;
+    a.seed = seed; a.step = step; a.chunk = 0;
     const int V = vector_width(ld, x, g, e, m, z);
     cudaError_t err = cudaSuccess;
     const int64_t body = n - n % V;

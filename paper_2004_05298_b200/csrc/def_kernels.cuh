@@ -129,6 +129,7 @@ struct StepArgs {
     float lambda;        // detach coefficient (used only when z is written)
     float delta;         // factor of the scaling compressor C(v) = delta v (used only by it)
     uint64_t seed, step; // the block start is drawn from these
+    int32_t chunk;       // stream kernel, chunked order: CTAs per row segment (see kOrderChunked)
 };
 
 // The start of this step's block, computed by one thread of the CTA and handed to the
@@ -291,17 +292,33 @@ __device__ __forceinline__ bool tile_touches_block(const StepArgs &a, int64_t s,
 // Consecutive CTAs sweep one row after the other, so the memory system sees a handful of
 // long sequential streams.  CTAs of tiles that touch the block leave at once.
 // With DETACH the kernel also writes z_w = x - lambda e'_w for its row (x is unchanged outside
-// the block).  WFAST then swaps the grid to (W, tiles): the W CTAs of a tile run together and
-// share one fetch of the tile's x from HBM, at the price of W interleaved row streams.
+// the block), which makes x a sixth stream that every worker's CTA of a tile reads.  ORDER
+// chooses how CTAs are numbered, i.e. what runs together:
+//   kOrderRows     grid (tiles, W): row after row, the flat stream.  (With DETACH, x would be
+//                  re-read from HBM for every row: it is far larger than the L2.)
+//   kOrderChunked  1-D grid: a.chunk consecutive CTAs sweep a segment of row 0, the next a.chunk
+//                  the same segment of row 1, ...; then the next segment.  Long sequential
+//                  streams, and the segment of x stays in the L2 until the last row has used it.
 // TILES CTAs' worth of tiles share one CTA of TILES * kTileThreads threads (each group of
 // kTileThreads threads still owns one tile and decides for it alone).
-template <bool MOM, int POL, bool DETACH = false, bool WFAST = false, int TILES = 1>
+constexpr int kOrderRows = 0, kOrderChunked = 1;
+
+template <bool MOM, int POL, bool DETACH = false, int ORDER = kOrderRows, int TILES = 1>
 __global__ void __launch_bounds__(kTileThreads * TILES)
 def_step_stream_kernel(const StepArgs a) {
     const int64_t s = cta_block_start(a);
-    const int64_t first = WFAST ? (int64_t)blockIdx.y + (int64_t)blockIdx.z * gridDim.y : (int64_t)blockIdx.x;
+    int64_t first;
+    unsigned w;
+    if (ORDER == kOrderRows) {
+        first = blockIdx.x; w = blockIdx.y;
+    } else {
+        const int64_t per_segment = (int64_t)a.W * a.chunk;
+        const int64_t segment = (int64_t)blockIdx.x / per_segment;
+        const int64_t rem = (int64_t)blockIdx.x - segment * per_segment;
+        w = (unsigned)(rem / a.chunk);
+        first = segment * a.chunk + rem % a.chunk;
+    }
     const int64_t tile = first * TILES + (int64_t)(threadIdx.x / kTileThreads);
-    const unsigned w = WFAST ? blockIdx.x : blockIdx.y;
     const int64_t col = tile * kTile + (int64_t)(threadIdx.x % kTileThreads) * 4;
     if (col >= a.n || tile_touches_block(a, s, tile)) return;
     const size_t at = (size_t)w * (size_t)a.ld + (size_t)col;

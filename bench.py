@@ -289,7 +289,7 @@ def bench_workload(B, WL, wl, steps, warmup, dist, world, rank, sampler=None, fl
 
 def bench_aux(B, WL, wl, reps=5):
     """Device time of the helpers around the step on the same workload: the detach point
-    (Algorithm 1 line 6), DEF's returned model and the distances of Eq. 9."""
+    (Algorithm 1's detach step), DEF's returned model and the distances of Eq. 9."""
     import torch
     dev = torch.device("cuda")
     W, d = wl.W, wl.d

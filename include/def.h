@@ -3,25 +3,25 @@
  *
  * One optimizer step of distributed momentum SGD with random block-wise gradient
  * sparsification (RBGS) under error feedback, from "Detached Error Feedback for
- * Distributed SGD with Random Sparsification": Algorithm 1 lines 7-10 with the
+ * Distributed SGD with Random Sparsification": Algorithm 1 from its error-feedback step to its update, with the
  * momentum substitution of Eq. 10, for W simulated workers (the paper's K) held as
  * the rows of [W, d] fp32 tensors on one GPU.  Per step and per worker w:
  *
  *     m'[w,j] = mu * m[w,j] + g[w,j]                          (Eq. 10)
- *     p[w,j]  = eta * m'[w,j] + e[w,j]                        (Eq. 10; Algorithm 1 line 7 when mu = 0)
+ *     p[w,j]  = eta * m'[w,j] + e[w,j]                        (Eq. 10; Algorithm 1's error-feedback step when mu = 0)
  *     C(p)    = p on the k block coordinates {(s+i) mod d}, 0 elsewhere   (Section 1, RBGS)
- *     e'[w,j] = p[w,j] - C(p)[w,j]                            (Algorithm 1 line 8)
- *     x[j]   -= (1/W) * sum_w C(p)[w,j]                       (Algorithm 1 lines 9-10)
+ *     e'[w,j] = p[w,j] - C(p)[w,j]                            (Algorithm 1's new-error step)
+ *     x[j]   -= (1/W) * sum_w C(p)[w,j]                       (Algorithm 1: ring-allreduce, update)
  *
  * The block start s is drawn once per step, the same for every worker (Section 1:
  * all workers hold the same seed), by a counter-based Philox4x32-10 generator keyed
- * by (seed, step).  The sum over workers stands in for the ring-allreduce of line 9;
+ * by (seed, step).  The sum over workers stands in for the algorithm's ring-allreduce;
  * it runs over w = 0..W-1 in that order in fp32, followed by an IEEE division by W.
  * Every product-and-add above is one fused multiply-add (one rounding).
  *
  * EF, DEF and DEF-A run the same step: they differ in where the caller evaluates
- * the gradient (Algorithm 1 line 6: at x_t - lambda e_{k,t}, lambda = 0 for EF) and
- * in the model that is returned after training (Algorithm 1's output line).
+ * the gradient (Algorithm 1's detach step: at x_t - lambda e_{k,t}, lambda = 0 for EF) and
+ * in the model that is returned after training (Algorithm 1's Output).
  *
  * Conventions
  *   - All tensors are fp32, row-major; [W, d] tensors are contiguous with row stride d
@@ -67,7 +67,7 @@ enum {
 /*
  * Algorithm 1's inputs.  d: model size; W: workers, 1..DEF_MAX_WORKERS; k: block
  * length, 1 <= k <= d (compression ratio d/k); variant: DEF_VARIANT_*; lr: eta,
- * finite; momentum: mu in [0, 1) (0 selects Algorithm 1 line 7 as printed);
+ * finite; momentum: mu in [0, 1) (0 selects Algorithm 1's error-feedback step as printed);
  * coeffs: NULL for the defaults {0.3, 0}, else coeffs[0] = lambda in [0, 1] (the
  * detach coefficient; forced to 0 for DEF_VARIANT_EF) and coeffs[1] = weight decay,
  * which must be 0 (the paper does not say where weight decay enters: fold it into
@@ -82,7 +82,7 @@ def_ctx *def_create(int64_t d, int32_t W, int64_t k, int32_t variant, float lr, 
 int def_destroy(def_ctx *ctx);
 
 /*
- * One step (Algorithm 1 lines 7-10, Eq. 10), in place.
+ * One step (Algorithm 1 from its error-feedback step to its update, Eq. 10), in place.
  *   params [d]     x_t      -> x_{t+1}   (only the k block coordinates are touched)
  *   grads  [W, d]  g_{k,t}     read only
  *   errors [W, d]  e_{k,t}  -> e_{k,t+1}
@@ -114,7 +114,7 @@ int def_step_columns(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, float *par
 
 /*
  * def_step / def_step_columns that also write where each worker evaluates its NEXT gradient
- * (Algorithm 1 line 6 of iteration t + 1), fused into the same two kernels:
+ * (Algorithm 1's detach step of iteration t + 1), fused into the same two kernels:
  *     detached_out[w, j] = x_{t+1}[j] - lambda * e_{w,t+1}[j]      (one fused multiply-add)
  * This is the one thing that makes DEF differ from plain EF at run time (EF, lambda = 0,
  * evaluates at x_{t+1} itself and has no use for it).  It costs one more [W, d] write:
@@ -129,16 +129,16 @@ int def_step_columns_detach(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, flo
 
 /*
  * The step with the WORKERS cut across GPUs (the paper's own deployment: one process per
- * GPU, each holding some of the K workers and a replica of the model; Algorithm 1 line 9 is
+ * GPU, each holding some of the K workers and a replica of the model; Algorithm 1's ring-allreduce step is
  * then a real all-reduce).  A context made with W = the number of LOCAL workers runs the step
  * in two halves around the caller's all-reduce:
- *   def_step_rows_local  lines 7-8 (Eq. 10) for the local rows, in place as in def_step, and
+ *   def_step_rows_local  the error-feedback and new-error steps (Eq. 10) for the local rows, in place as in def_step, and
  *                        block_sum_out[i] = sum over the local workers (in order) of C(p_w) at
  *                        block coordinate (s + i) mod d, i = 0..k-1: the k floats that travel.
  *                        params is not needed.
  *   (caller)             all-reduce(sum) of block_sum_out over the ranks -- additivity of the
  *                        compressor (Assumption 3) is what makes a plain sum valid.
- *   def_step_rows_apply  line 10: params[(s + i) mod d] -= block_sum[i] / W_total.
+ *   def_step_rows_apply  the update: params[(s + i) mod d] -= block_sum[i] / W_total.
  * Every rank passes the same (step, seed) and so cuts the same block.  With one rank the
  * result equals def_step bit for bit; with several, the order in which the all-reduce adds
  * the ranks' partial sums is the library's, so floats agree to rounding, not bitwise.
@@ -167,7 +167,7 @@ int def_step_columns_host(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, float
                           uint64_t step, uint64_t seed);
 
 /*
- * The point worker w evaluates its next gradient at (Algorithm 1 line 6):
+ * The point worker w evaluates its next gradient at (Algorithm 1's detach step):
  *     detached_out[w, j] = params[j] - lambda * errors[w, j]      (one fused multiply-add)
  * lambda is coeffs[0] of def_create (0 for DEF_VARIANT_EF, which makes every row a copy of
  * params).  View arguments as in def_step_columns: n coordinates, [W, n] tensors with row

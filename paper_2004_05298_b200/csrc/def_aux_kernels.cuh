@@ -1,5 +1,5 @@
-// Device code around the step: the detach point (Algorithm 1 line 6), the returned model
-// (Algorithm 1's output line) and the squared distances of Eq. 9.  All three are separate
+// Device code around the step: the detach point (Algorithm 1's detach step), the returned model
+// (Algorithm 1's Output) and the squared distances of Eq. 9.  All three are separate
 // per coordinate except for the final sum of the distances.
 #pragma once
 

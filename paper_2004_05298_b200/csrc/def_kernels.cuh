@@ -1,17 +1,17 @@
 // Device code of the DEF / DEF-A / EF step for sm_100a.
 //
-// The step (Algorithm 1 lines 7-10 with the momentum form of Eq. 10) is separate
+// The step (Algorithm 1 from its error-feedback step to its update, with the momentum form of Eq. 10) is separate
 // per model coordinate: a coordinate j needs g, m, e of its W workers and, if j is
 // one of the k block coordinates, x[j].  Two facts shape the kernels:
 //   * Outside the block nothing crosses workers (C(p) = 0, e' = p), so that part --
 //     all but k of the d coordinates -- is plain streaming of the [W, d] tensors and
 //     can be cut any way the memory system likes best.
 //   * On the block, the sum over workers that stands in for the ring-allreduce of
-//     line 9 is a register accumulation by one thread in the fixed order
+//     Algorithm 1 is a register accumulation by one thread in the fixed order
 //     w = 0..W-1: deterministic, with no shuffle, shared memory or atomics.
 // Either way g, m, e are read once and m', e' written once (20 bytes per gradient
 // element, the least the method can move) with 128-bit coalesced accesses, p never
-// goes to memory, and x is touched on the block only (line 10).  The block is a
+// goes to memory, and x is touched on the block only (Algorithm 1's update).  The block is a
 // predicate on j, never a slice: nothing is gathered or scattered.
 #pragma once
 
@@ -125,7 +125,7 @@ struct StepArgs {
     int32_t W;           // workers
     float eta;           // learning rate
     float mu;            // momentum constant
-    float W_float;       // (float)W, the divisor of line 9
+    float W_float;       // (float)W, the divisor of the average over workers
     float lambda;        // detach coefficient (used only when z is written)
     float delta;         // factor of the scaling compressor C(v) = delta v (used only by it)
     uint64_t seed, step; // the block start is drawn from these
@@ -142,7 +142,7 @@ __device__ __forceinline__ int64_t cta_block_start(const StepArgs &a) {
     return s_shared;
 }
 
-// One worker's row for V coordinates: Eq. 10 / line 7, then line 8.
+// One worker's row for V coordinates: Eq. 10 (or Algorithm 1's error-feedback step), then its new error.
 // `sent` accumulates C(p) over the workers in call order; `first` starts the sum.
 // SCALE selects the scaling compressor C(p) = delta p of the DEF-A paragraph (the case that
 // turns the iteration into SGD with iterate averaging, Eq. 11) instead of RBGS.
@@ -162,14 +162,14 @@ __device__ __forceinline__ void worker_row(const Vec<V> &g, const Vec<V> &m, con
         }
         const float c = SCALE ? __fmul_rn(delta, p) : (in[i] ? p : 0.0f);   // C(p)
         e_new.v[i] = __fsub_rn(p, c);                        // e' = p - C(p)
-        sent[i] = first ? c : __fadd_rn(sent[i], c);         // running sum of line 9
+        sent[i] = first ? c : __fadd_rn(sent[i], c);         // running sum over the workers
     }
 }
 
 // All W workers of the V coordinates starting at local coordinate `col`, in worker order,
-// U rows in flight at a time; then lines 9-10 on the coordinates that are in the block.
+// U rows in flight at a time; then the average and the update on the coordinates that are in the block.
 // With DETACH, a second walk over the rows writes the next iteration's gradient points
-// z_w = x_{t+1} - lambda e_{w,t+1} (Algorithm 1 line 6); it re-reads the e' this thread has
+// z_w = x_{t+1} - lambda e_{w,t+1} (Algorithm 1's detach step); it re-reads the e' this thread has
 // just written, which is still in cache.
 template <int V, bool MOM, int U, int POL, bool DETACH = false, bool SCALE = false>
 __device__ __forceinline__ void column_group(const StepArgs &a, int64_t s, int64_t col) {
@@ -219,7 +219,7 @@ __device__ __forceinline__ void column_group(const StepArgs &a, int64_t s, int64
 #pragma unroll
             for (int i = 0; i < V; ++i) {
                 if (in[i]) {
-                    if (a.block_sum) {                      // line 9 is finished by an all-reduce
+                    if (a.block_sum) {                      // the sum is finished by an all-reduce
                         int64_t o = off + i;
                         if (o >= a.d) o -= a.d;
                         a.block_sum[o] = sent[i];
@@ -372,7 +372,7 @@ def_step_block_kernel(const StepArgs a) {
     if (col < a.n) column_group<4, MOM, U, POL, DETACH>(a, s, col);
 }
 
-// Second half of a row-sharded step (Algorithm 1 lines 9-10 after the all-reduce):
+// Second half of a row-sharded step (Algorithm 1's update after the all-reduce):
 // x[(s + i) mod d] -= block_sum[i] / W_total for the k block coordinates.
 __global__ void __launch_bounds__(256)
 def_apply_block_kernel(float *__restrict__ x, const float *__restrict__ block_sum, StepArgs a) {

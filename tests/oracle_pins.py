@@ -128,7 +128,7 @@ def pin_full_block_is_momentum_sgd(o):
 
 
 # ---------------------------------------------------------------------------
-# Algorithm 1 line 8: C(p) + e' = p, coordinate by coordinate and bit for bit.
+# Algorithm 1's new-error step: C(p) + e' = p, coordinate by coordinate and bit for bit.
 # One worker, x_0 = 0, e_0 = 0, eta = 1, no momentum: then p = g exactly,
 # C(p) = -x_1 and e' = e_1.
 # ---------------------------------------------------------------------------
@@ -225,7 +225,7 @@ def pin_single_worker_lambda_one_is_sgd(o):
     e = np.zeros((1, d))
     theta = x.copy()                               # plain SGD iterate
     for t in range(T):
-        z = o.detach(x, e[0], 1.0)                 # Algorithm 1 line 6 with lambda = 1
+        z = o.detach(x, e[0], 1.0)                 # Algorithm 1's detach step with lambda = 1
         g = grad(z)[None, :]
         o.step(x, g, e, None, d=d, k=k, s=int(rng.integers(0, d)), eta=eta)
         theta = theta - eta * grad(theta)

@@ -1,5 +1,5 @@
-"""GPU parity of the helpers around the step -- the detach point (Algorithm 1 line 6), the
-returned model (Algorithm 1's output line) and the distances of Eq. 9 -- against the CPU
+"""GPU parity of the helpers around the step -- the detach point (Algorithm 1's detach step), the
+returned model (Algorithm 1's Output) and the distances of Eq. 9 -- against the CPU
 oracle, through the C boundary.  detach and output do the oracle's roundings in the oracle's
 order (bit-identical expected, gate 1e-5 relative).  The distances are fp64 sums whose
 order differs from the oracle's plain loop: for N = W * n summed terms the two can differ by

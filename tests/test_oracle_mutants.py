@@ -23,8 +23,8 @@ MUTANTS = [
     ("update_sign", "def_oracle_body.inc", "x[i] = x[i] - C_pt;", "x[i] = x[i] + C_pt;"),
     ("no_average", "def_oracle_body.inc", "REAL C_pt = sum / (REAL)W;", "REAL C_pt = sum;"),
     ("worker_dropped", "def_oracle_body.inc",
-     "for (int64_t w = 1; w < W; ++w)                     /* returns",
-     "for (int64_t w = 2; w < W; ++w)                     /* returns"),
+     "for (int64_t w = 1; w < W; ++w)                     /* workers added",
+     "for (int64_t w = 2; w < W; ++w)                     /* workers added"),
     ("momentum_operands_swapped", "def_oracle_body.inc",
      "m_w[i] = FMA(mu, m_w[i], g_w[i]);", "m_w[i] = FMA(mu, g_w[i], m_w[i]);"),
     ("momentum_not_used_in_p", "def_oracle_body.inc",

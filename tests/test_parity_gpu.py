@@ -415,7 +415,7 @@ def test_stream_and_resume(B):
 
 
 # ---------------------------------------------------------------------------
-# the step with the fused detach output (Algorithm 1 line 6 of the next iteration)
+# the step with the fused detach output (Algorithm 1's detach step of the next iteration)
 # ---------------------------------------------------------------------------
 def run_detach(B, d, W, k, steps, momentum, lam, variant=0, offsets=(0, 0, 0, 0, 0), seed=7, pair=True):
     dev = torch.device("cuda")

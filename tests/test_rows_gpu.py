@@ -1,4 +1,4 @@
-"""The row-sharded step (workers cut across GPUs, Algorithm 1 line 9 as a real all-reduce) on
+"""The row-sharded step (workers cut across GPUs, Algorithm 1's ring-allreduce step as a real all-reduce) on
 ONE GPU: with a one-rank NCCL group it must equal def_step bit for bit; with two ranks'
 halves run one after the other and their block sums added, it must equal the oracle's step
 over all workers up to the order in which the workers' values are added."""

@@ -82,7 +82,7 @@ def test_shard_columns_partition():
 
 
 # ---------------------------------------------------------------------------
-# Row sharding: workers cut across ranks, Algorithm 1 line 9 as an all-reduce (gloo, CPU).
+# Row sharding: workers cut across ranks, Algorithm 1's ring-allreduce step as an all-reduce (gloo, CPU).
 # Each rank gets the sum of its own workers' sparsified vectors from the oracle (a step from
 # x = 0 with eta-scaled inputs moves x by minus their mean; two workers per rank keep the
 # mean's scaling exact), the ranks all-reduce those sums, and every rank applies the average.

@@ -39,7 +39,7 @@ FALLBACK_HBM_GBS = 6650.0
 # hash of the kernel source the capture was taken on.  Reported only while the source is
 # unchanged (see profiles/).
 NCU_TRAFFIC_BYTES_PER_ELEMENT = 19.42
-NCU_TRAFFIC_KERNEL_SHA256 = "7b81ddec9953dca1cada36a392c78c28ebc0eed5aea00ea46c9086dd5d12274c"
+NCU_TRAFFIC_KERNEL_SHA256 = "ea1d10fafd7aa50e17c08906966e4120c90e3eb586b0b4f56c1051c4d7b4ad07"
 
 
 def _measured_peak():

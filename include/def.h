@@ -89,10 +89,10 @@ int def_destroy(def_ctx *ctx);
  *   mom    [W, d]  m_{k,t}  -> m_{k,t+1}; NULL if and only if momentum == 0
  *   step, seed     t and the shared seed: the block start is a pure function of both
  * The caller zeroes errors and mom before step 0 (Algorithm 1's initialisation).
- * 16-byte aligned pointers with d % 4 == 0 run on 128-bit accesses (the fast path); 8-byte /
- * d % 2 and 4-byte alignment are accepted and run on narrower accesses, 6 % and 14 % slower at
- * large sizes.  A model whose d is not a multiple of 4 keeps the fast path by padding its
- * rows: allocate [W, ld] with ld = d rounded up to 4 and call def_step_columns(ctx, 0, d, ld, ...).
+ * 16-byte aligned base pointers run on 128-bit accesses whatever d is (when d % 4 != 0 the
+ * rows themselves are unaligned and the contiguous [W, d] tensors are streamed flat, 1.5 %
+ * slower); bases that are only 8- or 4-byte aligned are accepted and run on narrower accesses,
+ * 6 % and 14 % slower at large sizes.
  * Errors: DEF_ERR_NULL, DEF_ERR_ALIGN, DEF_ERR_ALIAS (any two of the four tensors
  * overlap), DEF_ERR_DEVICE, DEF_ERR_CUDA (launch failure).
  */

@@ -258,6 +258,28 @@ int enqueue_columns(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, float *x, c
     a.seed = seed; a.step = step; a.chunk = 0;
     const int V = vector_width(ld, x, g, e, m, z);
     cudaError_t err = cudaSuccess;
+    // Contiguous rows that are not 16-byte aligned but whose bases are: block coordinates by one
+    // kernel, everything else as a flat stream that ignores the row boundaries.
+    const bool flat_ok = V < 4 && ld == n && n >= defk::kFlatTile && !z && !block_sum &&
+                         ctx->compressor == DEF_COMPRESSOR_RBGS &&
+                         (((uintptr_t)g | (uintptr_t)e | (uintptr_t)m) & 15u) == 0 &&
+                         20 * (int64_t)ctx->W * n >= ctx->small_step_bytes;
+    if (flat_ok) {
+        const int64_t block_grid = (ctx->k + 255) / 256;
+        const int64_t flat_grid = ((int64_t)ctx->W * n + defk::kFlatTile - 1) / defk::kFlatTile;
+        if (block_grid > 0x7fffffffLL || flat_grid > 0x7fffffffLL) return fail(DEF_ERR_ARG, "problem too large for one grid");
+        err = counted_launch(ctx, DEF_KERNEL_BLOCK, stream, [&] {
+            if (m) defk::def_step_block_columns_kernel<true, 8, kPolicy><<<(unsigned)block_grid, 256, 0, stream>>>(a);
+            else defk::def_step_block_columns_kernel<false, 8, kPolicy><<<(unsigned)block_grid, 256, 0, stream>>>(a);
+        });
+        if (err != cudaSuccess) return cuda_fail(err, "def_step block-columns kernel launch");
+        err = counted_launch(ctx, DEF_KERNEL_STREAM, stream, [&] {
+            if (m) defk::def_step_flat_kernel<true, kPolicy><<<(unsigned)flat_grid, defk::kFlatThreads, 0, stream>>>(a);
+            else defk::def_step_flat_kernel<false, kPolicy><<<(unsigned)flat_grid, defk::kFlatThreads, 0, stream>>>(a);
+        });
+        if (err != cudaSuccess) return cuda_fail(err, "def_step flat kernel launch");
+        return DEF_OK;
+    }
     const int64_t body = n - n % V;
     if (body > 0) {
         a.n = body;

@@ -372,6 +372,92 @@ def_step_block_kernel(const StepArgs a) {
     if (col < a.n) column_group<4, MOM, U, POL, DETACH>(a, s, col);
 }
 
+// ---------------------------------------------------------------------------
+// Contiguous [W, n] tensors whose rows are NOT 16-byte aligned (n % 4 != 0) but whose bases
+// are: the part outside the block is still a plain stream, so it is run flat over the W * n
+// floats with 16-byte accesses that ignore the row boundaries; every float finds its own
+// (worker, coordinate) and skips itself if the coordinate is in the block.  The block
+// coordinates -- exactly k of them -- are done beforehand by def_step_block_columns_kernel,
+// one thread per coordinate walking the W rows in order with 4-byte accesses.
+// ---------------------------------------------------------------------------
+constexpr int kFlatThreads = 512;
+constexpr int64_t kFlatTile = (int64_t)kFlatThreads * 4;     // floats per CTA; needs n >= kFlatTile
+
+template <bool MOM, int U, int POL>
+__global__ void __launch_bounds__(256)
+def_step_block_columns_kernel(const StepArgs a) {
+    const int64_t s = cta_block_start(a);
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;   // i-th block coordinate
+    if (i >= a.k) return;
+    int64_t j = s + i;
+    if (j >= a.d) j -= a.d;
+    const int64_t col = j - a.j0;
+    if (col >= 0 && col < a.n) column_group<1, MOM, U, POL>(a, s, col);
+}
+
+template <bool MOM, int POL>
+__global__ void __launch_bounds__(kFlatThreads)
+def_step_flat_kernel(const StepArgs a) {
+    __shared__ int64_t shared[3];
+    const int64_t total = (int64_t)a.W * a.n;                 // rows are contiguous: ld == n
+    const int64_t base = (int64_t)blockIdx.x * kFlatTile;
+    if (threadIdx.x == 0) {
+        shared[0] = block_start(a.seed, a.step, a.d);
+        shared[1] = base / a.n;                               // worker of the CTA's first float
+        shared[2] = base - shared[1] * a.n;                   // and its coordinate
+    }
+    __syncthreads();
+    const int64_t s = shared[0];
+    const int64_t f = base + (int64_t)threadIdx.x * 4;
+    if (f >= total) return;
+    int64_t c = shared[2] + (int64_t)threadIdx.x * 4;        // < 2 n because n >= kFlatTile
+    if (c >= a.n) c -= a.n;
+    bool in[4];
+    bool any = false;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        int64_t ci = c + i;                                   // coordinate of float f + i (next row after a wrap)
+        if (ci >= a.n) ci -= a.n;
+        int64_t off = a.j0 + ci - s;
+        if (off < 0) off += a.d;
+        in[i] = off < a.k;
+        any |= in[i];
+    }
+    const bool none[4] = {false, false, false, false};
+    float unused[4];
+    if (f + 4 <= total) {
+        const Vec<4> g = load_vec<4, POL>(a.g + f);
+        const Vec<4> e = load_vec<4, POL>(a.e + f);
+        Vec<4> m, m_new, e_new;
+        if (MOM) m = load_vec<4, POL>(a.m + f);
+        worker_row<4, MOM>(g, m, e, none, a.eta, a.mu, true, m_new, e_new, unused);
+        if (!any) {
+            if (MOM) store_vec<4, POL>(a.m + f, m_new);
+            store_vec<4, POL>(a.e + f, e_new);
+        } else {                                              // leave the block's floats to the other kernel
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                if (!in[i]) {
+                    if (MOM) a.m[f + i] = m_new.v[i];
+                    a.e[f + i] = e_new.v[i];
+                }
+            }
+        }
+    } else {                                                  // the last W * n % 4 floats
+        for (int i = 0; f + i < total; ++i) {
+            if (in[i]) continue;
+            Vec<1> g, e, m, m_new, e_new;
+            g.v[0] = a.g[f + i]; e.v[0] = a.e[f + i];
+            if (MOM) m.v[0] = a.m[f + i];
+            const bool no[1] = {false};
+            float u1[1];
+            worker_row<1, MOM>(g, m, e, no, a.eta, a.mu, true, m_new, e_new, u1);
+            if (MOM) a.m[f + i] = m_new.v[0];
+            a.e[f + i] = e_new.v[0];
+        }
+    }
+}
+
 // Second half of a row-sharded step (Algorithm 1's update after the all-reduce):
 // x[(s + i) mod d] -= block_sum[i] / W_total for the k block coordinates.
 __global__ void __launch_bounds__(256)

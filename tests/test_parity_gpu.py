@@ -573,3 +573,31 @@ def test_step_replays_from_a_cuda_graph(B, pair):
         oracle.step(xo, gh, eo, mo, d=d, k=k, s=s, eta=0.1, mu=0.9)
     assert np.array_equal(x.cpu().numpy(), xo) and np.array_equal(e.cpu().numpy(), eo) and np.array_equal(m.cpu().numpy(), mo)
     B.def_destroy(ctx)
+
+
+@pytest.mark.parametrize("d", [5_000_001, 3_000_002, 2_051])
+def test_unaligned_contiguous_rows_take_the_flat_path(B, d):
+    """d % 4 != 0 with 16-byte aligned bases: block coordinates by one kernel, the rest as a flat
+    stream over the W * d floats.  Whole tensors against the oracle, wrapped blocks included."""
+    dev = torch.device("cuda")
+    W, k, seed = 7, max(1, d // 16), 12
+    rng = np.random.default_rng(d)
+    x = torch.from_numpy((0.05 * rng.standard_normal(d)).astype(np.float32)).to(dev)
+    e = torch.zeros(W, d, device=dev); m = torch.zeros(W, d, device=dev)
+    xo = x.cpu().numpy().copy(); eo = np.zeros((W, d), np.float32); mo = np.zeros((W, d), np.float32)
+    ctx = B.def_create(d, W, k, 0, 0.1, 0.9)
+    B.def_set_small_step_bytes(ctx, 0)
+    B.def_set_kernel_timing(ctx, True)
+    steps = [0, 1] + find_steps(d, k, seed, lambda s: s + k > d)[:1]
+    for t in steps:
+        gh = (0.1 * rng.standard_normal((W, d))).astype(np.float32)
+        g = torch.from_numpy(gh).to(dev)
+        B.def_step(ctx, x, g, e, m, t, seed)
+        oracle.step(xo, gh, eo, mo, d=d, k=k, s=oracle.block_start(seed, t, d), eta=0.1, mu=0.9)
+        assert torch.equal(g.cpu(), torch.from_numpy(gh))
+    assert B.def_kernel_time(ctx, B.DEF_KERNEL_STREAM)[1] == len(steps)
+    assert B.def_kernel_time(ctx, B.DEF_KERNEL_BLOCK)[1] == len(steps)
+    assert B.def_kernel_time(ctx, B.DEF_KERNEL_GENERAL)[1] == 0
+    assert np.array_equal(x.cpu().numpy(), xo)
+    assert np.array_equal(e.cpu().numpy(), eo) and np.array_equal(m.cpu().numpy(), mo)
+    B.def_destroy(ctx)

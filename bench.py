@@ -39,7 +39,7 @@ FALLBACK_HBM_GBS = 6650.0
 # hash of the kernel source the capture was taken on.  Reported only while the source is
 # unchanged (see profiles/).
 NCU_TRAFFIC_BYTES_PER_ELEMENT = 19.42
-NCU_TRAFFIC_KERNEL_SHA256 = "ea1d10fafd7aa50e17c08906966e4120c90e3eb586b0b4f56c1051c4d7b4ad07"
+NCU_TRAFFIC_KERNEL_SHA256 = "b6e0a0d95cae0553fba88743673f9a3663075c8a188aee55a700bc54f144e78a"
 
 
 def _measured_peak():

@@ -35,6 +35,9 @@
  *   - Every function returns DEF_OK (0) or a negative DEF_ERR_* code and leaves a
  *     human-readable message for def_last_error() (thread-local).  Nothing is
  *     launched when validation fails.  No exception crosses this boundary.
+ *   - A def_ctx is not internally locked: use it from one host thread at a time (different
+ *     contexts are independent).  Work enqueued by successive calls on one stream runs in
+ *     call order; tensors must stay valid until that work has run.
  *   - IEEE specials in the data propagate as the arithmetic above dictates; inputs are
  *     not scanned.
  */

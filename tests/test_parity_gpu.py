@@ -601,3 +601,24 @@ def test_unaligned_contiguous_rows_take_the_flat_path(B, d):
     assert np.array_equal(x.cpu().numpy(), xo)
     assert np.array_equal(e.cpu().numpy(), eo) and np.array_equal(m.cpu().numpy(), mo)
     B.def_destroy(ctx)
+
+
+def test_random_shapes_and_layouts(B):
+    """Seeded sweep over shapes, alignments, launch strategies, momentum on/off and the fused
+    detach output: every case bit-identical to the oracle, nothing written outside the tensors."""
+    rng = np.random.default_rng(20260101)
+    for case in range(60):
+        d = int(rng.choice([rng.integers(1, 40), rng.integers(40, 5000), rng.integers(5000, 60000)]))
+        W = int(rng.choice([1, 2, 3, 5, 8, 16, 33]))
+        k = int(rng.choice([1, d, max(1, d // 2), int(rng.integers(1, d + 1))]))
+        momentum = float(rng.choice([0.0, 0.5, 0.9]))
+        offsets = tuple(int(v) for v in rng.integers(0, 4, size=5))
+        if rng.random() < 0.5:
+            offsets = (0, 0, 0, 0, 0)
+        pair = bool(rng.integers(0, 2))
+        seed = int(rng.integers(0, 1000))
+        steps = [int(v) for v in rng.integers(0, 10 ** 6, size=3)]
+        if rng.random() < 0.4:
+            run_detach(B, d, W, k, steps, momentum, float(rng.choice([0.0, 0.3, 1.0])), offsets=offsets, seed=seed, pair=pair)
+        else:
+            assert run_whole(B, d, W, k, steps, momentum, seed, offsets=offsets[:4], pair=pair), (case, d, W, k)

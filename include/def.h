@@ -257,11 +257,11 @@ enum { DEF_COMPRESSOR_RBGS = 0, DEF_COMPRESSOR_SCALE = 1 };
 int def_set_compressor(def_ctx *ctx, int32_t compressor, float delta);
 
 /*
- * Launch strategy of a step on 16-byte aligned rows.  A step that moves at least `bytes`
- * (20 * W * n) runs as the block + stream kernel pair, which is what reaches HBM speed; a
- * smaller one is bound by launch latency and runs as one launch of the general kernel.
- * Default 1 GiB (the measured crossover on B200); 0 always uses the pair.  Results are
- * bit-identical either way.
+ * Launch strategy of a step whose tensors start on 16-byte boundaries.  A step that moves at
+ * least `bytes` (20 * W * n) runs as a pair of kernels (block coordinates, then everything else
+ * as a stream that is allowed to start beside the first); a smaller one runs as one launch of
+ * the general kernel.  Default 128 MiB: below that a step is bound by the launches themselves
+ * when run back to back; 0 always uses the pair.  Results are bit-identical either way.
  */
 int def_set_small_step_bytes(def_ctx *ctx, int64_t bytes);
 

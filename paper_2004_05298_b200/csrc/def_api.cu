@@ -172,6 +172,27 @@ cudaError_t counted_launch(def_ctx *ctx, int kind, cudaStream_t stream, Launch l
     return cudaSuccess;
 }
 
+// Launch of the stream kernel right after the block kernel of the same step.  The two work on
+// disjoint tiles, so the stream kernel is allowed to start while the block kernel still runs
+// (programmatic stream serialization; the block kernel releases its dependents at once).  That
+// hides the block kernel's latency-bound run on mid-sized models.  Everything launched later
+// still waits for both kernels, as usual in a stream.  Not used in timing mode, where each
+// kernel is measured alone.
+template <typename Kernel>
+cudaError_t launch_beside_block_kernel(const def_ctx *ctx, Kernel kernel, dim3 grid, unsigned threads,
+                                       cudaStream_t stream, const defk::StepArgs &a) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(threads);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = ctx->timing ? 0 : 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, a);
+}
+
 // With the fused detach output x becomes a stream every worker's CTA of a tile reads.  The
 // stream kernel then runs in chunked order: 256 CTAs (two tiles each: 2 MB of every row and
 // of x) sweep a segment of row 0, the next 256 the same segment of row 1, and so on, so the
@@ -180,11 +201,15 @@ cudaError_t counted_launch(def_ctx *ctx, int kind, cudaStream_t stream, Launch l
 // adjacent and 8.97 ms row after row (x re-read from HBM for every row).
 constexpr int kDetachChunkCtas = 256;
 
-// Below about this many bytes of [W, n] traffic a step is bound by launch and ramp-up latency,
-// not by bandwidth, and one launch of the general kernel beats the block + stream pair
-// (measured with a flushed L2: 19.5 vs 25.6 us at 80 MB, 54.5 vs 58.4 us at 320 MB, 286.8 vs
-// 283.7 us at 1.9 GB).  def_set_small_step_bytes changes it per context.
-constexpr int64_t kSmallStepBytesDefault = (int64_t)1 << 30;
+// Steps that move fewer bytes than this run as ONE launch of the general kernel instead of the
+// kernel pair.  With the stream kernel allowed to start beside the block kernel the pair is at
+// least as fast from cold memory at every size measured (flushed L2: 13.3 vs 14.3 us at 40 MB,
+// 19.5 vs 20.4 us at 80 MB, 27.6 vs 28.7 us on the 137 MB ResNet-56-sized workload, 275 vs 287 us
+// at 1.9 GB); only tiny models stepped back to back out of the L2 are bound by the launches
+// themselves and prefer one (7.4 vs 9.4 us at 40 MB, 10.4 vs 10.8 us at 80 MB; the pair leads
+// from 160 MB).  Hence 128 MiB.
+// def_set_small_step_bytes changes it per context.
+constexpr int64_t kSmallStepBytesDefault = (int64_t)128 << 20;
 
 template <int V, bool MOM, bool DETACH>
 cudaError_t launch_one(def_ctx *ctx, const defk::StepArgs &a, cudaStream_t stream) {
@@ -216,8 +241,8 @@ cudaError_t launch_one(def_ctx *ctx, const defk::StepArgs &a, cudaStream_t strea
             defk::StepArgs c = a;
             c.chunk = kDetachChunkCtas;
             return counted_launch(ctx, DEF_KERNEL_STREAM, stream, [&] {
-                defk::def_step_stream_kernel<MOM, kPolicy, true, defk::kOrderChunked, kStreamTiles>
-                    <<<(unsigned)ctas, defk::kTileThreads * kStreamTiles, 0, stream>>>(c);
+                launch_beside_block_kernel(ctx, defk::def_step_stream_kernel<MOM, kPolicy, true, defk::kOrderChunked, kStreamTiles>,
+                                           dim3((unsigned)ctas), defk::kTileThreads * kStreamTiles, stream, c);
             });
         }
         else {
@@ -225,8 +250,8 @@ cudaError_t launch_one(def_ctx *ctx, const defk::StepArgs &a, cudaStream_t strea
             // many block-start computations), while 1024 threads lose 20 %
             const dim3 grid((unsigned)slots, (unsigned)a.W);
             return counted_launch(ctx, DEF_KERNEL_STREAM, stream, [&] {
-                defk::def_step_stream_kernel<MOM, kPolicy, false, defk::kOrderRows, kStreamTiles>
-                    <<<grid, defk::kTileThreads * kStreamTiles, 0, stream>>>(a);
+                launch_beside_block_kernel(ctx, defk::def_step_stream_kernel<MOM, kPolicy, false, defk::kOrderRows, kStreamTiles>,
+                                           grid, defk::kTileThreads * kStreamTiles, stream, a);
             });
         }
     }
@@ -274,8 +299,8 @@ int enqueue_columns(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, float *x, c
         });
         if (err != cudaSuccess) return cuda_fail(err, "def_step block-columns kernel launch");
         err = counted_launch(ctx, DEF_KERNEL_STREAM, stream, [&] {
-            if (m) defk::def_step_flat_kernel<true, kPolicy><<<(unsigned)flat_grid, defk::kFlatThreads, 0, stream>>>(a);
-            else defk::def_step_flat_kernel<false, kPolicy><<<(unsigned)flat_grid, defk::kFlatThreads, 0, stream>>>(a);
+            if (m) launch_beside_block_kernel(ctx, defk::def_step_flat_kernel<true, kPolicy>, dim3((unsigned)flat_grid), defk::kFlatThreads, stream, a);
+            else launch_beside_block_kernel(ctx, defk::def_step_flat_kernel<false, kPolicy>, dim3((unsigned)flat_grid), defk::kFlatThreads, stream, a);
         });
         if (err != cudaSuccess) return cuda_fail(err, "def_step flat kernel launch");
         return DEF_OK;

@@ -349,6 +349,10 @@ def_step_stream_kernel(const StepArgs a) {
 template <bool MOM, int U, int POL, bool DETACH = false>
 __global__ void __launch_bounds__(kTileThreads)
 def_step_block_kernel(const StepArgs a) {
+    // The stream kernel that follows in the stream works on other tiles and needs nothing from
+    // this kernel: when it was launched with programmatic stream serialization, let its CTAs
+    // start now instead of after this grid has drained (a no-op otherwise).
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int64_t s = cta_block_start(a);
     // the two runs in model coordinates, clipped to the local range [j0, j0 + n)
     const int64_t lo = a.j0, hi = a.j0 + a.n;
@@ -386,6 +390,9 @@ constexpr int64_t kFlatTile = (int64_t)kFlatThreads * 4;     // floats per CTA; 
 template <bool MOM, int U, int POL>
 __global__ void __launch_bounds__(256)
 def_step_block_columns_kernel(const StepArgs a) {
+    // the flat kernel that follows touches no float of a block coordinate: let it start now
+    // when it was launched with programmatic stream serialization
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int64_t s = cta_block_start(a);
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;   // i-th block coordinate
     if (i >= a.k) return;
@@ -423,38 +430,36 @@ def_step_flat_kernel(const StepArgs a) {
         in[i] = off < a.k;
         any |= in[i];
     }
-    const bool none[4] = {false, false, false, false};
-    float unused[4];
-    if (f + 4 <= total) {
+    bool all = true;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) all &= in[i];
+    if (all) return;                                          // the block's floats belong to the other kernel
+    if (!any && f + 4 <= total) {
+        const bool none[4] = {false, false, false, false};
+        float unused[4];
         const Vec<4> g = load_vec<4, POL>(a.g + f);
         const Vec<4> e = load_vec<4, POL>(a.e + f);
         Vec<4> m, m_new, e_new;
         if (MOM) m = load_vec<4, POL>(a.m + f);
         worker_row<4, MOM>(g, m, e, none, a.eta, a.mu, true, m_new, e_new, unused);
-        if (!any) {
-            if (MOM) store_vec<4, POL>(a.m + f, m_new);
-            store_vec<4, POL>(a.e + f, e_new);
-        } else {                                              // leave the block's floats to the other kernel
+        if (MOM) store_vec<4, POL>(a.m + f, m_new);
+        store_vec<4, POL>(a.e + f, e_new);
+        return;
+    }
+    // a group that straddles an edge of the block, or the last W * n % 4 floats: float by float,
+    // touching nothing that is in the block
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                if (!in[i]) {
-                    if (MOM) a.m[f + i] = m_new.v[i];
-                    a.e[f + i] = e_new.v[i];
-                }
-            }
-        }
-    } else {                                                  // the last W * n % 4 floats
-        for (int i = 0; f + i < total; ++i) {
-            if (in[i]) continue;
-            Vec<1> g, e, m, m_new, e_new;
-            g.v[0] = a.g[f + i]; e.v[0] = a.e[f + i];
-            if (MOM) m.v[0] = a.m[f + i];
-            const bool no[1] = {false};
-            float u1[1];
-            worker_row<1, MOM>(g, m, e, no, a.eta, a.mu, true, m_new, e_new, u1);
-            if (MOM) a.m[f + i] = m_new.v[0];
-            a.e[f + i] = e_new.v[0];
-        }
+    for (int i = 0; i < 4; ++i) {
+        if (in[i] || f + i >= total) continue;
+        Vec<1> g, e, m, m_new, e_new;
+        g.v[0] = a.g[f + i];
+        e.v[0] = a.e[f + i];
+        if (MOM) m.v[0] = a.m[f + i];
+        const bool no[1] = {false};
+        float u1[1];
+        worker_row<1, MOM>(g, m, e, no, a.eta, a.mu, true, m_new, e_new, u1);
+        if (MOM) a.m[f + i] = m_new.v[0];
+        a.e[f + i] = e_new.v[0];
     }
 }
 

@@ -125,8 +125,7 @@ def run_whole(B, d, W, k, steps, momentum, seed, lr=0.1, offsets=(0, 0, 0, 0), s
     x64 = xo.astype(np.float64); e64 = eo.astype(np.float64)
     m64 = mo.astype(np.float64) if momentum else None
     ctx = B.def_create(d, W, k, variant, lr, momentum)
-    if pair:
-        B.def_set_small_step_bytes(ctx, 0)          # the block + stream kernel pair even at this size
+    B.def_set_small_step_bytes(ctx, 0 if pair else 1 << 60)   # the kernel pair, or one launch of the general kernel
     exact = True
     for t in steps:
         gh = (sigma * rng.standard_normal((W, d))).astype(np.float32)
@@ -345,8 +344,7 @@ def test_step_columns_equals_whole_step(B, pair):
     cuts = [0, 4, 70_000, 70_003, 150_002, d]                     # aligned and unaligned pieces
     xs = [x[a:b].clone() for a, b in zip(cuts[:-1], cuts[1:])]
     ctx = B.def_create(d, W, k, wl.variant, wl.lr, wl.momentum)
-    if pair:
-        B.def_set_small_step_bytes(ctx, 0)
+    B.def_set_small_step_bytes(ctx, 0 if pair else 1 << 60)
     es = [torch.zeros(W, b - a + 5, device=dev) for a, b in zip(cuts[:-1], cuts[1:])]   # ld = n + 5
     ms = [torch.zeros(W, b - a + 5, device=dev) for a, b in zip(cuts[:-1], cuts[1:])]
     for t in range(6):
@@ -431,8 +429,7 @@ def run_detach(B, d, W, k, steps, momentum, lam, variant=0, offsets=(0, 0, 0, 0,
     xo = x.cpu().numpy().copy(); eo = np.zeros((W, d), np.float32)
     mo = np.zeros((W, d), np.float32) if momentum else None
     ctx = B.def_create(d, W, k, variant, 0.1, momentum, (lam, 0.0))
-    if pair:
-        B.def_set_small_step_bytes(ctx, 0)
+    B.def_set_small_step_bytes(ctx, 0 if pair else 1 << 60)
     lam_used = 0.0 if variant == B.DEF_VARIANT_EF else lam
     for t in steps:
         gh = (0.1 * rng.standard_normal((W, d))).astype(np.float32)
@@ -554,8 +551,7 @@ def test_step_replays_from_a_cuda_graph(B, pair):
     e = torch.zeros(W, d, device=dev); m = torch.zeros(W, d, device=dev)
     xo = x.cpu().numpy().copy(); eo = np.zeros((W, d), np.float32); mo = np.zeros((W, d), np.float32)
     ctx = B.def_create(d, W, k, 0, 0.1, 0.9)
-    if pair:
-        B.def_set_small_step_bytes(ctx, 0)
+    B.def_set_small_step_bytes(ctx, 0 if pair else 1 << 60)
     B.def_step(ctx, x, g, e, m, 5, 3)                      # first call outside capture (device query)
     graph = torch.cuda.CUDAGraph()
     side = torch.cuda.Stream()

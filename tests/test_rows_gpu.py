@@ -40,8 +40,7 @@ def test_one_rank_nccl_group_equals_def_step(B, pair):
     try:
         wl = WL.get(1).scaled(300_004, W=5)
         ctx = B.def_create(wl.d, wl.W, wl.k, 0, wl.lr, wl.momentum)
-        if pair:
-            B.def_set_small_step_bytes(ctx, 0)
+        B.def_set_small_step_bytes(ctx, 0 if pair else 1 << 60)
         x1 = WL.initial_params(wl, dev); e1, m1 = WL.zeros_state(wl, dev)
         x2 = x1.clone(); e2, m2 = WL.zeros_state(wl, dev)
         block = torch.full((wl.k,), 7.0, device=dev)

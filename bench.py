@@ -4,7 +4,7 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
 A step is one pass of the whole hot path (block start, momentum, error feedback,
-sparsification, cross-worker average, update: one fused kernel launch) over one batch
+sparsification, cross-worker average, update: two kernels that run side by side) over one batch
 of synthetic gradients.  The timed workload is the VGG-16-sized one (d = 138,357,544,
 W = 16, k = d/32, DEF, momentum 0.9): its 35 GB of state and gradients are far larger
 than the L2, so no flush is needed between iterations.  Prints ONE JSON line on rank 0.

@@ -43,7 +43,8 @@ def _offset_view(t, offset):
     return v
 
 
-@pytest.mark.parametrize("d,W", [(1, 1), (7, 3), (4096, 4), (100_003, 5), (262_146, 16), (50_000, 64)])
+@pytest.mark.parametrize("d,W", [(1, 1), (7, 3), (4096, 4), (100_003, 5), (262_146, 16), (50_000, 64), (262_144, 16),
+                                 (131_072, 3), (1_000_000, 5)])
 @pytest.mark.parametrize("offset", [0, 1, 2])
 def test_detach_and_output(B, d, W, offset):
     for variant, lam in ((B.DEF_VARIANT_DEF, 0.3), (B.DEF_VARIANT_DEF_A, 1.0), (B.DEF_VARIANT_EF, 0.7)):
@@ -64,8 +65,9 @@ def test_detach_and_output(B, d, W, offset):
         B.def_destroy(ctx)
 
 
-def test_views_with_padding(B):
-    d, W, n, ld = 10_000, 4, 3_001, 3_006
+@pytest.mark.parametrize("d,n,ld", [(10_000, 3_001, 3_006), (400_000, 131_072, 131_080)])
+def test_views_with_padding(B, d, n, ld):
+    W = 4
     ctx, x, e = _state(d, W, 2, B)
     el = torch.full((W, ld), 9.0, device="cuda"); el[:, :n] = e[:, 100:100 + n]
     xl = x[100:100 + n].clone()

@@ -325,6 +325,21 @@ def bench_aux(B, WL, wl, reps=5):
         ms = a.elapsed_time(b) / reps
         out.append({"op": name, "ms": ms, "algorithmic_bytes": nbytes, "GB/s": nbytes / (ms * 1e-3) / 1e9})
     B.def_destroy(ctx)
+    # Algorithm 1 as printed, without the momentum buffers: 12 B per gradient element
+    ctx0 = B.def_create(d, W, wl.k, WL.VARIANT_DEF, wl.lr, 0.0, (wl.lam, 0.0))
+    for t in range(3):
+        B.def_step(ctx0, x, g, e, None, t, wl.rbgs_seed)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for t in range(reps):
+        B.def_step(ctx0, x, g, e, None, 3 + t, wl.rbgs_seed)
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / reps
+    nbytes = 12 * W * d + 8 * wl.k
+    out.append({"op": "def_step without momentum", "ms": ms, "algorithmic_bytes": nbytes, "GB/s": nbytes / (ms * 1e-3) / 1e9})
+    B.def_destroy(ctx0)
     del x, e, z, y, g, m
     torch.cuda.empty_cache()
     return out

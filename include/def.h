@@ -145,12 +145,47 @@ int def_step_columns_detach(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, flo
  * Every rank passes the same (step, seed) and so cuts the same block.  With one rank the
  * result equals def_step bit for bit; with several, the order in which the all-reduce adds
  * the ranks' partial sums is the library's, so floats agree to rounding, not bitwise.
- * RBGS only (DEF_ERR_UNSUPPORTED under DEF_COMPRESSOR_SCALE).  Whole model (n = ld = d).
+ * RBGS only (DEF_ERR_UNSUPPORTED under DEF_COMPRESSOR_SCALE).  Whole model (n = ld = d); any d
+ * (16-byte aligned bases keep 128-bit accesses when d % 4 != 0, as in def_step).
  */
 int def_step_rows_local(def_ctx *ctx, const float *grads, float *errors, float *mom,
                         float *block_sum_out, uint64_t step, uint64_t seed);
 int def_step_rows_apply(def_ctx *ctx, float *params, const float *block_sum, int32_t W_total,
                         uint64_t step, uint64_t seed);
+
+/*
+ * The row-sharded step that also writes where each LOCAL worker evaluates its next gradient
+ * (Algorithm 1's detach step of iteration t + 1; see def_step_detach), still at one extra
+ * [W, d] write.  Outside the block x does not change in this step, so the local half already
+ * knows z[w, j] = x_t[j] - lambda * e_{w,t+1}[j]; it reads params [d] for that and does not
+ * write it.  On the k block coordinates e_{w,t+1} = +0, so z[w, j] = x_{t+1}[j], which exists
+ * only after the all-reduce: the local half leaves x_t[j] there and def_step_rows_apply_detach
+ * overwrites those k floats of every local row when it updates params.  After the pair of
+ * calls detached_out [W, d] equals what def_step_detach would have written for these workers.
+ * detached_out must overlap none of the other tensors.
+ */
+int def_step_rows_local_detach(def_ctx *ctx, const float *params, const float *grads, float *errors,
+                               float *mom, float *block_sum_out, float *detached_out, uint64_t step,
+                               uint64_t seed);
+int def_step_rows_apply_detach(def_ctx *ctx, float *params, const float *block_sum, int32_t W_total,
+                               float *detached_out, uint64_t step, uint64_t seed);
+
+/*
+ * Takes the all-reduce of a row-sharded step off the critical path.  The k block sums are ready
+ * as soon as the few tiles that touch the block are done, long before the rest of the [W, d]
+ * tensors has been streamed.  With a side stream set (a cudaStream_t other than the context's
+ * stream; NULL switches back), def_step_rows_local[_detach] makes the side stream wait for what
+ * the context's stream holds so far, runs the kernel of the block tiles THERE and everything
+ * else on the context's stream as before; the caller enqueues its all-reduce of block_sum_out on
+ * the side stream; def_step_rows_apply[_detach] runs there too, and then makes the context's
+ * stream wait for it.  The collective and the update so overlap the streaming kernel, and work
+ * enqueued on the context's stream after the apply call sees the finished step.  (Steps that run
+ * as a single kernel -- models under the def_set_small_step_bytes threshold, bases that are not
+ * 16-byte aligned -- produce the sums on the context's stream; the side stream is then made to
+ * wait for that kernel, so the same calling sequence stays correct.)  The first non-NULL call
+ * creates two events.  The caller owns the stream and keeps it alive while it is set.
+ */
+int def_set_rows_stream(def_ctx *ctx, void *side_stream);
 
 /*
  * One step with every tensor in HOST memory (pinned memory is much faster; pageable

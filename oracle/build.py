@@ -12,6 +12,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 SOURCES = ["def_oracle.c"]
 DEPENDS = ["def_oracle.c", "def_oracle_body.inc"]
 LIB = os.path.join(HERE, "libdef_oracle.so")
+LIB_ALL_CORES = os.path.join(HERE, "libdef_oracle_allcores.so")   # same source, coordinate loops as OpenMP parallel-for
 CFLAGS = ["-O2", "-std=c11", "-fPIC", "-shared", "-ffp-contract=off", "-fno-fast-math",
           "-Wall", "-Wextra"]
 
@@ -25,7 +26,7 @@ def needs_build(lib=LIB):
 
 def build(force=False, lib=LIB, source_dir=HERE, extra_flags=()):
     """gcc the oracle; returns the path of the shared library."""
-    if not force and lib == LIB and not needs_build(lib):
+    if not force and lib in (LIB, LIB_ALL_CORES) and not needs_build(lib):
         return lib
     tmp = lib + ".tmp.%d" % os.getpid()
     cmd = ["gcc", *CFLAGS, *extra_flags, "-I", source_dir,
@@ -35,5 +36,11 @@ def build(force=False, lib=LIB, source_dir=HERE, extra_flags=()):
     return lib
 
 
+def build_all_cores(force=False):
+    """The same source with -fopenmp: the loops over coordinates become parallel-for loops."""
+    return build(force=force, lib=LIB_ALL_CORES, extra_flags=("-fopenmp",))
+
+
 if __name__ == "__main__":
     print(build(force=True))
+    print(build_all_cores(force=True))

@@ -115,6 +115,13 @@ void def_oracle_block_mask(int64_t d, int64_t k, int64_t s, int64_t n, const int
     }
 }
 
+/* Loops over coordinates: serial here; a parallel-for in the all-cores build (see the body). */
+#ifdef _OPENMP
+#define FOR_EACH_COORDINATE _Pragma("omp parallel for schedule(static)")
+#else
+#define FOR_EACH_COORDINATE
+#endif
+
 #define REAL float
 #define FMA fmaf
 #define NAME(base) base##_f32
@@ -130,3 +137,14 @@ void def_oracle_block_mask(int64_t d, int64_t k, int64_t s, int64_t n, const int
 #undef REAL
 #undef FMA
 #undef NAME
+
+/* Threads the coordinate loops run on: 1 in the plain build. */
+int def_oracle_threads(void)
+{
+#ifdef _OPENMP
+    extern int omp_get_max_threads(void);
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}

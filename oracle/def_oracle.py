@@ -17,7 +17,7 @@ VARIANT_EF = 2
 
 __all__ = [
     "COMPRESSOR_RBGS", "COMPRESSOR_SCALE", "VARIANT_DEF", "VARIANT_DEF_A", "VARIANT_EF",
-    "Oracle", "default", "philox4x32", "block_start", "in_block", "block_mask", "compress",
+    "Oracle", "default", "all_cores", "philox4x32", "block_start", "in_block", "block_mask", "compress",
     "step", "detach", "output", "stats",
 ]
 
@@ -62,6 +62,8 @@ class Oracle:
         lib.def_oracle_in_block.restype = ctypes.c_int
         lib.def_oracle_block_mask.argtypes = [_i64, _i64, _i64, _i64, _ptr, _ptr]
         lib.def_oracle_block_mask.restype = None
+        lib.def_oracle_threads.argtypes = []
+        lib.def_oracle_threads.restype = ctypes.c_int
         for sfx, real in (("f32", ctypes.c_float), ("f64", ctypes.c_double)):
             f = getattr(lib, "def_oracle_compress_" + sfx)
             f.argtypes = [ctypes.c_int, _i64, _i64, _i64, real, _i64, _ptr, _ptr, _ptr]
@@ -79,6 +81,10 @@ class Oracle:
             f = getattr(lib, "def_oracle_stats_" + sfx)
             f.argtypes = [real, _i64, _i64, _ptr, _ptr]
             f.restype = None
+
+    def threads(self):
+        """Host threads the loops over coordinates run on (1 unless this is the all-cores build)."""
+        return int(self.lib.def_oracle_threads())
 
     # ---- block start ------------------------------------------------------
     def philox4x32(self, ctr, key, rounds=10):
@@ -181,6 +187,18 @@ def default():
     if _default is None:
         _default = Oracle()
     return _default
+
+
+_all_cores = None
+
+
+def all_cores():
+    """The same source built with OpenMP: loops over coordinates run on every host core, with
+    the operations on each coordinate and their order unchanged (same bits as default())."""
+    global _all_cores
+    if _all_cores is None:
+        _all_cores = Oracle(_build.build_all_cores())
+    return _all_cores
 
 
 def philox4x32(ctr, key, rounds=10):

@@ -30,6 +30,9 @@ SIGNATURES = {
     "def_step_columns_detach": (ctypes.c_int, [_ptr, _i64, _i64, _i64, _ptr, _ptr, _ptr, _ptr, _ptr, _u64, _u64]),
     "def_step_rows_local": (ctypes.c_int, [_ptr, _ptr, _ptr, _ptr, _ptr, _u64, _u64]),
     "def_step_rows_apply": (ctypes.c_int, [_ptr, _ptr, _ptr, _i32, _u64, _u64]),
+    "def_step_rows_local_detach": (ctypes.c_int, [_ptr, _ptr, _ptr, _ptr, _ptr, _ptr, _ptr, _u64, _u64]),
+    "def_step_rows_apply_detach": (ctypes.c_int, [_ptr, _ptr, _ptr, _i32, _ptr, _u64, _u64]),
+    "def_set_rows_stream": (ctypes.c_int, [_ptr, _ptr]),
     "def_step_host": (ctypes.c_int, [_ptr, _ptr, _ptr, _ptr, _ptr, _u64, _u64]),
     "def_step_columns_host": (ctypes.c_int, [_ptr, _i64, _i64, _i64, _ptr, _ptr, _ptr, _ptr, _u64, _u64]),
     "def_detach": (ctypes.c_int, [_ptr, _i64, _i64, _ptr, _ptr, _ptr]),
@@ -286,10 +289,46 @@ def def_step_rows_apply(ctx, params, block_sum, W_total, step, seed):
                                    _dev(block_sum, "block_sum", (ctx.k,)), int(W_total), int(step), int(seed)))
 
 
-def def_step_rows(ctx, params, grads, errors, mom, block_sum, step, seed, group=None):
+def def_step_rows_local_detach(ctx, params, grads, errors, mom, block_sum_out, detached_out, step, seed):
+    d, W = ctx.d, ctx.W
+    _check(lib.def_step_rows_local_detach(ctx.handle, _dev(params, "params", (d,)), _dev(grads, "grads", (W, d)),
+                                          _dev(errors, "errors", (W, d)), _dev(mom, "mom", (W, d), optional=True),
+                                          _dev(block_sum_out, "block_sum_out", (ctx.k,)),
+                                          _dev(detached_out, "detached_out", (W, d)), int(step), int(seed)))
+
+
+def def_step_rows_apply_detach(ctx, params, block_sum, W_total, detached_out, step, seed):
+    _check(lib.def_step_rows_apply_detach(ctx.handle, _dev(params, "params", (ctx.d,)),
+                                          _dev(block_sum, "block_sum", (ctx.k,)), int(W_total),
+                                          _dev(detached_out, "detached_out", (ctx.W, ctx.d)), int(step), int(seed)))
+
+
+def def_set_rows_stream(ctx, stream):
+    """Side stream of the row-sharded step (a torch.cuda.Stream, or None to switch it off): the
+    block kernel, the all-reduce and the update run there, beside the streaming kernel."""
+    raw = stream.cuda_stream if isinstance(stream, torch.cuda.Stream) else (stream or 0)
+    _check(lib.def_set_rows_stream(ctx.handle, ctypes.c_void_p(raw)))
+    ctx.rows_stream = stream if isinstance(stream, torch.cuda.Stream) else None
+
+
+def def_step_rows(ctx, params, grads, errors, mom, block_sum, step, seed, group=None, detached_out=None):
     """One row-sharded step: local half, all-reduce of the k block sums over `group` (NCCL through
-    torch.distributed, on the current stream), apply.  W_total = local W times the group size."""
+    torch.distributed), apply.  W_total = local W times the group size.  After def_set_rows_stream
+    the all-reduce is issued on that side stream, where the library has put the block kernel and
+    puts the update, so that it overlaps the streaming kernel on the context's stream."""
     import torch.distributed as dist
-    def_step_rows_local(ctx, grads, errors, mom, block_sum, step, seed)
-    dist.all_reduce(block_sum, op=dist.ReduceOp.SUM, group=group)
-    def_step_rows_apply(ctx, params, block_sum, ctx.W * dist.get_world_size(group), step, seed)
+    if detached_out is None:
+        def_step_rows_local(ctx, grads, errors, mom, block_sum, step, seed)
+    else:
+        def_step_rows_local_detach(ctx, params, grads, errors, mom, block_sum, detached_out, step, seed)
+    side = getattr(ctx, "rows_stream", None)
+    if side is not None:
+        with torch.cuda.stream(side):
+            dist.all_reduce(block_sum, op=dist.ReduceOp.SUM, group=group)
+    else:
+        dist.all_reduce(block_sum, op=dist.ReduceOp.SUM, group=group)
+    W_total = ctx.W * dist.get_world_size(group)
+    if detached_out is None:
+        def_step_rows_apply(ctx, params, block_sum, W_total, step, seed)
+    else:
+        def_step_rows_apply_detach(ctx, params, block_sum, W_total, detached_out, step, seed)

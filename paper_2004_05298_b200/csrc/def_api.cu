@@ -59,6 +59,12 @@ struct def_ctx {
     int sm_count = 0;
     // def_stats: per-CTA partial sums (allocated by the first def_stats call)
     double *stats_scratch = nullptr;
+    // row-sharded step: the caller's side stream for the block kernel, the all-reduce and the
+    // update (def_set_rows_stream), the events that fork it from and join it to `stream`, and
+    // whether the last local half left block sums behind on `stream` itself
+    cudaStream_t rows_stream = nullptr;
+    cudaEvent_t rows_fork = nullptr, rows_join = nullptr;
+    bool sums_on_main = false;
     // host-memory path
     bool host_ready = false;
     int64_t host_chunk = 0;  // coordinates per staging slot (multiple of 4)
@@ -175,19 +181,21 @@ cudaError_t counted_launch(def_ctx *ctx, int kind, cudaStream_t stream, Launch l
 // Launch of the stream kernel right after the block kernel of the same step.  The two work on
 // disjoint tiles, so the stream kernel is allowed to start while the block kernel still runs
 // (programmatic stream serialization; the block kernel releases its dependents at once).  That
-// hides the block kernel's latency-bound run on mid-sized models.  Everything launched later
-// still waits for both kernels, as usual in a stream.  Not used in timing mode, where each
-// kernel is measured alone.
+// hides the block kernel's latency-bound run on mid-sized models.  The stream kernel's threads
+// end with a wait for the block kernel's grid, so whatever is enqueued later, being ordered
+// behind the stream kernel, is ordered behind both.  Not used in timing mode, where each
+// kernel is measured alone, nor when the block kernel went to another stream (`beside` false:
+// the two then overlap as work on two streams does).
 template <typename Kernel>
 cudaError_t launch_beside_block_kernel(const def_ctx *ctx, Kernel kernel, dim3 grid, unsigned threads,
-                                       cudaStream_t stream, const defk::StepArgs &a) {
+                                       cudaStream_t stream, const defk::StepArgs &a, bool beside = true) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = dim3(threads);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = ctx->timing ? 0 : 1;
+    attr[0].val.programmaticStreamSerializationAllowed = (ctx->timing || !beside) ? 0 : 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, a);
@@ -211,8 +219,11 @@ constexpr int kDetachChunkCtas = 256;
 // def_set_small_step_bytes changes it per context.
 constexpr int64_t kSmallStepBytesDefault = (int64_t)128 << 20;
 
+// `block_stream`: where the kernel of the tiles that touch the block goes when the step runs as a
+// pair (the row-sharded step puts it on a side stream so that the all-reduce of the block sums
+// can follow it there while the stream kernel runs); equal to `stream` otherwise.
 template <int V, bool MOM, bool DETACH>
-cudaError_t launch_one(def_ctx *ctx, const defk::StepArgs &a, cudaStream_t stream) {
+cudaError_t launch_one(def_ctx *ctx, const defk::StepArgs &a, cudaStream_t stream, cudaStream_t block_stream) {
     const int64_t groups = a.n / V;
     if (groups == 0) return cudaSuccess;
     if (ctx->compressor == DEF_COMPRESSOR_SCALE) {   // dense: every coordinate is sent and updated
@@ -228,8 +239,9 @@ cudaError_t launch_one(def_ctx *ctx, const defk::StepArgs &a, cudaStream_t strea
         // the few tiles that touch the block first, then the stream over all the others
         const int64_t block_ctas = a.k / defk::kTile + 4;
         const unsigned block_grid = (unsigned)(block_ctas < tiles + 1 ? block_ctas : tiles + 1);
-        cudaError_t err = counted_launch(ctx, DEF_KERNEL_BLOCK, stream, [&] {
-            defk::def_step_block_kernel<MOM, kBlockRows, kPolicy, DETACH><<<block_grid, defk::kTileThreads, 0, stream>>>(a);
+        const bool beside = block_stream == stream;
+        cudaError_t err = counted_launch(ctx, DEF_KERNEL_BLOCK, block_stream, [&] {
+            defk::def_step_block_kernel<MOM, kBlockRows, kPolicy, DETACH><<<block_grid, defk::kTileThreads, 0, block_stream>>>(a);
         });
         if (err != cudaSuccess) return err;
         constexpr int kStreamTiles = 2;
@@ -242,7 +254,7 @@ cudaError_t launch_one(def_ctx *ctx, const defk::StepArgs &a, cudaStream_t strea
             c.chunk = kDetachChunkCtas;
             return counted_launch(ctx, DEF_KERNEL_STREAM, stream, [&] {
                 launch_beside_block_kernel(ctx, defk::def_step_stream_kernel<MOM, kPolicy, true, defk::kOrderChunked, kStreamTiles>,
-                                           dim3((unsigned)ctas), defk::kTileThreads * kStreamTiles, stream, c);
+                                           dim3((unsigned)ctas), defk::kTileThreads * kStreamTiles, stream, c, beside);
             });
         }
         else {
@@ -251,7 +263,7 @@ cudaError_t launch_one(def_ctx *ctx, const defk::StepArgs &a, cudaStream_t strea
             const dim3 grid((unsigned)slots, (unsigned)a.W);
             return counted_launch(ctx, DEF_KERNEL_STREAM, stream, [&] {
                 launch_beside_block_kernel(ctx, defk::def_step_stream_kernel<MOM, kPolicy, false, defk::kOrderRows, kStreamTiles>,
-                                           grid, defk::kTileThreads * kStreamTiles, stream, a);
+                                           grid, defk::kTileThreads * kStreamTiles, stream, a, beside);
             });
         }
     }
@@ -260,22 +272,24 @@ cudaError_t launch_one(def_ctx *ctx, const defk::StepArgs &a, cudaStream_t strea
     const int64_t want = (groups + kThreads - 1) / kThreads;
     const int64_t cap = 0x7fffffffLL;
     const unsigned grid = (unsigned)(want < cap ? want : cap);
+    if (a.block_sum) ctx->sums_on_main = true;
     return counted_launch(ctx, DEF_KERNEL_GENERAL, stream, [&] {
         defk::def_step_kernel<V, MOM, 4, DETACH><<<grid, kThreads, 0, stream>>>(a);
     });
 }
 
 template <int V>
-cudaError_t launch_v(def_ctx *ctx, const defk::StepArgs &a, cudaStream_t stream) {
-    if (a.z) return a.m ? launch_one<V, true, true>(ctx, a, stream) : launch_one<V, false, true>(ctx, a, stream);
-    return a.m ? launch_one<V, true, false>(ctx, a, stream) : launch_one<V, false, false>(ctx, a, stream);
+cudaError_t launch_v(def_ctx *ctx, const defk::StepArgs &a, cudaStream_t stream, cudaStream_t block_stream) {
+    if (a.z) return a.m ? launch_one<V, true, true>(ctx, a, stream, block_stream) : launch_one<V, false, true>(ctx, a, stream, block_stream);
+    return a.m ? launch_one<V, true, false>(ctx, a, stream, block_stream) : launch_one<V, false, false>(ctx, a, stream, block_stream);
 }
 
 // Enqueue the step on local coordinates [0, n) of a view; counts launches.
 int enqueue_columns(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, float *x, const float *g,
                     float *e, float *m, uint64_t step, uint64_t seed, cudaStream_t stream,
-                    float *z = nullptr, float *block_sum = nullptr) {
+                    float *z = nullptr, float *block_sum = nullptr, cudaStream_t block_stream = nullptr) {
     if (n == 0) return DEF_OK;
+    if (!block_sum || !block_stream) block_stream = stream;
     defk::StepArgs a;
     a.x = x; a.g = g; a.e = e; a.m = m; a.z = z; a.block_sum = block_sum; a.lambda = ctx->lambda; a.delta = ctx->delta;
     a.n = n; a.ld = ld; a.d = ctx->d; a.j0 = j0; a.k = ctx->k; a.W = ctx->W;
@@ -285,7 +299,7 @@ int enqueue_columns(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, float *x, c
     cudaError_t err = cudaSuccess;
     // Contiguous rows that are not 16-byte aligned but whose bases are: block coordinates by one
     // kernel, everything else as a flat stream that ignores the row boundaries.
-    const bool flat_ok = V < 4 && ld == n && n >= defk::kFlatTile && !z && !block_sum &&
+    const bool flat_ok = V < 4 && ld == n && n >= defk::kFlatTile && !z &&
                          ctx->compressor == DEF_COMPRESSOR_RBGS &&
                          (((uintptr_t)g | (uintptr_t)e | (uintptr_t)m) & 15u) == 0 &&
                          20 * (int64_t)ctx->W * n >= ctx->small_step_bytes;
@@ -293,14 +307,15 @@ int enqueue_columns(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, float *x, c
         const int64_t block_grid = (ctx->k + 255) / 256;
         const int64_t flat_grid = ((int64_t)ctx->W * n + defk::kFlatTile - 1) / defk::kFlatTile;
         if (block_grid > 0x7fffffffLL || flat_grid > 0x7fffffffLL) return fail(DEF_ERR_ARG, "problem too large for one grid");
-        err = counted_launch(ctx, DEF_KERNEL_BLOCK, stream, [&] {
-            if (m) defk::def_step_block_columns_kernel<true, 8, kPolicy><<<(unsigned)block_grid, 256, 0, stream>>>(a);
-            else defk::def_step_block_columns_kernel<false, 8, kPolicy><<<(unsigned)block_grid, 256, 0, stream>>>(a);
+        const bool beside = block_stream == stream;
+        err = counted_launch(ctx, DEF_KERNEL_BLOCK, block_stream, [&] {
+            if (m) defk::def_step_block_columns_kernel<true, 8, kPolicy><<<(unsigned)block_grid, 256, 0, block_stream>>>(a);
+            else defk::def_step_block_columns_kernel<false, 8, kPolicy><<<(unsigned)block_grid, 256, 0, block_stream>>>(a);
         });
         if (err != cudaSuccess) return cuda_fail(err, "def_step block-columns kernel launch");
         err = counted_launch(ctx, DEF_KERNEL_STREAM, stream, [&] {
-            if (m) launch_beside_block_kernel(ctx, defk::def_step_flat_kernel<true, kPolicy>, dim3((unsigned)flat_grid), defk::kFlatThreads, stream, a);
-            else launch_beside_block_kernel(ctx, defk::def_step_flat_kernel<false, kPolicy>, dim3((unsigned)flat_grid), defk::kFlatThreads, stream, a);
+            if (m) launch_beside_block_kernel(ctx, defk::def_step_flat_kernel<true, kPolicy>, dim3((unsigned)flat_grid), defk::kFlatThreads, stream, a, beside);
+            else launch_beside_block_kernel(ctx, defk::def_step_flat_kernel<false, kPolicy>, dim3((unsigned)flat_grid), defk::kFlatThreads, stream, a, beside);
         });
         if (err != cudaSuccess) return cuda_fail(err, "def_step flat kernel launch");
         return DEF_OK;
@@ -308,8 +323,8 @@ int enqueue_columns(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, float *x, c
     const int64_t body = n - n % V;
     if (body > 0) {
         a.n = body;
-        err = V == 4 ? launch_v<4>(ctx, a, stream) : V == 2 ? launch_v<2>(ctx, a, stream)
-                                                              : launch_v<1>(ctx, a, stream);
+        err = V == 4 ? launch_v<4>(ctx, a, stream, block_stream) : V == 2 ? launch_v<2>(ctx, a, stream, block_stream)
+                                                                            : launch_v<1>(ctx, a, stream, block_stream);
         if (err != cudaSuccess) return cuda_fail(err, "def_step kernel launch");
     }
     if (body < n) {  // the last n % V coordinates, one float at a time
@@ -317,7 +332,7 @@ int enqueue_columns(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, float *x, c
         t.x = x + body; t.g = g + body; t.e = e + body; t.m = m ? m + body : nullptr;
         t.z = z ? z + body : nullptr;
         t.n = n - body; t.j0 = j0 + body;
-        err = launch_v<1>(ctx, t, stream);
+        err = launch_v<1>(ctx, t, stream, block_stream);
         if (err != cudaSuccess) return cuda_fail(err, "def_step tail kernel launch");
     }
     return DEF_OK;
@@ -431,6 +446,8 @@ int def_destroy(def_ctx *ctx) {
     if (!ctx) return fail(DEF_ERR_NULL, "ctx is NULL");
     free_host_path(ctx);
     if (ctx->stats_scratch) cudaFree(ctx->stats_scratch);
+    if (ctx->rows_fork) cudaEventDestroy(ctx->rows_fork);
+    if (ctx->rows_join) cudaEventDestroy(ctx->rows_join);
     if (ctx->t_begin) cudaEventDestroy(ctx->t_begin);
     if (ctx->t_end) cudaEventDestroy(ctx->t_end);
     delete ctx;
@@ -439,6 +456,8 @@ int def_destroy(def_ctx *ctx) {
 
 int def_set_stream(def_ctx *ctx, void *cuda_stream) {
     if (!ctx) return fail(DEF_ERR_NULL, "ctx is NULL");
+    if (ctx->rows_stream && (void *)ctx->rows_stream == cuda_stream)
+        return fail(DEF_ERR_ARG, "the context's stream must differ from its side stream");
     ctx->stream = (cudaStream_t)cuda_stream;
     return DEF_OK;
 }
@@ -664,49 +683,139 @@ int def_step_detach(def_ctx *ctx, float *params, const float *grads, float *erro
     return def_step_columns_detach(ctx, 0, ctx->d, ctx->d, params, grads, errors, mom, detached_out, step, seed);
 }
 
-int def_step_rows_local(def_ctx *ctx, const float *grads, float *errors, float *mom,
-                        float *block_sum_out, uint64_t step, uint64_t seed) {
+}  // extern "C"
+
+namespace {
+
+// First half of a row-sharded step; `params` and `z` are both NULL (plain) or both set (with the
+// detach output).
+int rows_local(def_ctx *ctx, const float *params, const float *grads, float *errors, float *mom,
+               float *block_sum_out, float *z, uint64_t step, uint64_t seed) {
     if (!ctx) return fail(DEF_ERR_NULL, "ctx is NULL");
     if (ctx->compressor != DEF_COMPRESSOR_RBGS)
         return fail(DEF_ERR_UNSUPPORTED, "row-sharded steps support the RBGS compressor only");
     if (!block_sum_out) return fail(DEF_ERR_NULL, "block_sum_out must not be NULL");
     if ((uintptr_t)block_sum_out & 3u) return fail(DEF_ERR_ALIGN, "block_sum_out is not 4-byte aligned");
-    // params is not touched by the local half; validate the rest as usual (block_sum_out takes
-    // the place of params in the overlap checks, with its own length k)
     if (!grads || !errors) return fail(DEF_ERR_NULL, "grads and errors must not be NULL");
     if (ctx->momentum != 0.f && !mom) return fail(DEF_ERR_NULL, "mom must not be NULL when momentum != 0");
     if (ctx->momentum == 0.f && mom) return fail(DEF_ERR_ARG, "mom must be NULL when momentum == 0");
     if (((uintptr_t)grads | (uintptr_t)errors | (uintptr_t)mom) & 3u) return fail(DEF_ERR_ALIGN, "a tensor is not 4-byte aligned");
     const size_t rows_b = span_rows(ctx->W, ctx->d, ctx->d), bs_b = (size_t)ctx->k * sizeof(float);
+    const size_t x_b = (size_t)ctx->d * sizeof(float);
     if (overlaps(grads, rows_b, errors, rows_b) || (mom && (overlaps(mom, rows_b, errors, rows_b) || overlaps(mom, rows_b, grads, rows_b))))
         return fail(DEF_ERR_ALIAS, "grads, errors and mom must not overlap");
     if (overlaps(block_sum_out, bs_b, grads, rows_b) || overlaps(block_sum_out, bs_b, errors, rows_b) ||
         (mom && overlaps(block_sum_out, bs_b, mom, rows_b)))
         return fail(DEF_ERR_ALIAS, "block_sum_out overlaps a tensor");
+    if (z) {
+        if (!params) return fail(DEF_ERR_NULL, "params must not be NULL");
+        if ((uintptr_t)params & 3u) return fail(DEF_ERR_ALIGN, "params is not 4-byte aligned");
+        if (overlaps(params, x_b, grads, rows_b) || overlaps(params, x_b, errors, rows_b) ||
+            (mom && overlaps(params, x_b, mom, rows_b)) || overlaps(params, x_b, block_sum_out, bs_b))
+            return fail(DEF_ERR_ALIAS, "params overlaps another tensor");
+        int rc = validate_detach_out(ctx, ctx->d, ctx->d, z, params, grads, errors, mom);
+        if (rc != DEF_OK) return rc;
+        if (overlaps(z, rows_b, block_sum_out, bs_b)) return fail(DEF_ERR_ALIAS, "detached_out overlaps block_sum_out");
+    }
     int rc = check_device(ctx);
     if (rc != DEF_OK) return rc;
-    // x is never dereferenced when block_sum is set; the errors pointer stands in for the alignment class
-    return enqueue_columns(ctx, 0, ctx->d, ctx->d, errors, grads, errors, mom, step, seed, ctx->stream, nullptr, block_sum_out);
+    cudaStream_t side = ctx->rows_stream;
+    cudaError_t err;
+    ctx->sums_on_main = false;
+    if (side) {
+        // The side stream picks up where `stream` is now: behind the previous step's kernels and
+        // whatever produced the gradients.  The block kernel then runs there, beside the stream
+        // kernel on `stream`, and the caller's all-reduce can follow it without waiting for the latter.
+        if ((err = cudaEventRecord(ctx->rows_fork, ctx->stream)) != cudaSuccess ||
+            (err = cudaStreamWaitEvent(side, ctx->rows_fork, 0)) != cudaSuccess)
+            return cuda_fail(err, "forking the side stream");
+    }
+    // Without the detach output x is never dereferenced by the local half (block_sum is set); the
+    // errors pointer stands in for the alignment class.
+    float *x_arg = z ? const_cast<float *>(params) : errors;
+    rc = enqueue_columns(ctx, 0, ctx->d, ctx->d, x_arg, grads, errors, mom, step, seed, ctx->stream, z, block_sum_out, side);
+    if (rc != DEF_OK) return rc;
+    if (side && ctx->sums_on_main) {   // a kernel on `stream` wrote block sums: the side stream must see them
+        if ((err = cudaEventRecord(ctx->rows_fork, ctx->stream)) != cudaSuccess ||
+            (err = cudaStreamWaitEvent(side, ctx->rows_fork, 0)) != cudaSuccess)
+            return cuda_fail(err, "ordering the side stream behind the step kernel");
+    }
+    return DEF_OK;
+}
+
+int rows_apply(def_ctx *ctx, float *params, const float *block_sum, int32_t W_total, float *z,
+               uint64_t step, uint64_t seed) {
+    if (!ctx) return fail(DEF_ERR_NULL, "ctx is NULL");
+    if (!params || !block_sum) return fail(DEF_ERR_NULL, "params and block_sum must not be NULL");
+    if (((uintptr_t)params | (uintptr_t)block_sum | (uintptr_t)z) & 3u) return fail(DEF_ERR_ALIGN, "a pointer is not 4-byte aligned");
+    if (W_total < ctx->W) return fail(DEF_ERR_ARG, "W_total=%d is smaller than this context's W=%d", W_total, ctx->W);
+    const size_t x_b = (size_t)ctx->d * sizeof(float), bs_b = (size_t)ctx->k * sizeof(float);
+    if (overlaps(params, x_b, block_sum, bs_b)) return fail(DEF_ERR_ALIAS, "params and block_sum overlap");
+    if (z) {
+        const size_t rows_b = span_rows(ctx->W, ctx->d, ctx->d);
+        if (overlaps(z, rows_b, params, x_b) || overlaps(z, rows_b, block_sum, bs_b))
+            return fail(DEF_ERR_ALIAS, "detached_out overlaps params or block_sum");
+    }
+    int rc = check_device(ctx);
+    if (rc != DEF_OK) return rc;
+    defk::StepArgs a = {};
+    a.d = ctx->d; a.ld = ctx->d; a.k = ctx->k; a.W = W_total; a.W_float = (float)W_total; a.seed = seed; a.step = step;
+    const int64_t blocks = (ctx->k + 255) / 256;
+    if (blocks > 0x7fffffffLL) return fail(DEF_ERR_ARG, "k too large");
+    cudaStream_t side = ctx->rows_stream;
+    cudaStream_t run = side ? side : ctx->stream;
+    defk::def_apply_block_kernel<<<(unsigned)blocks, 256, 0, run>>>(params, block_sum, z, ctx->W, a);
+    cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) return cuda_fail(err, "def_step_rows_apply kernel launch");
+    ctx->launches += 1;
+    if (side) {   // `stream` goes on only when the side stream's part of the step is done
+        if ((err = cudaEventRecord(ctx->rows_join, side)) != cudaSuccess ||
+            (err = cudaStreamWaitEvent(ctx->stream, ctx->rows_join, 0)) != cudaSuccess)
+            return cuda_fail(err, "joining the side stream");
+    }
+    return DEF_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int def_step_rows_local(def_ctx *ctx, const float *grads, float *errors, float *mom,
+                        float *block_sum_out, uint64_t step, uint64_t seed) {
+    return rows_local(ctx, nullptr, grads, errors, mom, block_sum_out, nullptr, step, seed);
 }
 
 int def_step_rows_apply(def_ctx *ctx, float *params, const float *block_sum, int32_t W_total,
                         uint64_t step, uint64_t seed) {
+    return rows_apply(ctx, params, block_sum, W_total, nullptr, step, seed);
+}
+
+int def_step_rows_local_detach(def_ctx *ctx, const float *params, const float *grads, float *errors,
+                               float *mom, float *block_sum_out, float *detached_out, uint64_t step,
+                               uint64_t seed) {
+    if (!detached_out) return fail(DEF_ERR_NULL, "detached_out must not be NULL");
+    if (!params) return fail(DEF_ERR_NULL, "params must not be NULL");
+    return rows_local(ctx, params, grads, errors, mom, block_sum_out, detached_out, step, seed);
+}
+
+int def_step_rows_apply_detach(def_ctx *ctx, float *params, const float *block_sum, int32_t W_total,
+                               float *detached_out, uint64_t step, uint64_t seed) {
+    if (!detached_out) return fail(DEF_ERR_NULL, "detached_out must not be NULL");
+    return rows_apply(ctx, params, block_sum, W_total, detached_out, step, seed);
+}
+
+int def_set_rows_stream(def_ctx *ctx, void *side_stream) {
     if (!ctx) return fail(DEF_ERR_NULL, "ctx is NULL");
-    if (!params || !block_sum) return fail(DEF_ERR_NULL, "params and block_sum must not be NULL");
-    if (((uintptr_t)params | (uintptr_t)block_sum) & 3u) return fail(DEF_ERR_ALIGN, "a pointer is not 4-byte aligned");
-    if (W_total < ctx->W) return fail(DEF_ERR_ARG, "W_total=%d is smaller than this context's W=%d", W_total, ctx->W);
-    if (overlaps(params, (size_t)ctx->d * sizeof(float), block_sum, (size_t)ctx->k * sizeof(float)))
-        return fail(DEF_ERR_ALIAS, "params and block_sum overlap");
-    int rc = check_device(ctx);
-    if (rc != DEF_OK) return rc;
-    defk::StepArgs a = {};
-    a.d = ctx->d; a.k = ctx->k; a.W = W_total; a.W_float = (float)W_total; a.seed = seed; a.step = step;
-    const int64_t blocks = (ctx->k + 255) / 256;
-    if (blocks > 0x7fffffffLL) return fail(DEF_ERR_ARG, "k too large");
-    defk::def_apply_block_kernel<<<(unsigned)blocks, 256, 0, ctx->stream>>>(params, block_sum, a);
-    cudaError_t err = cudaGetLastError();
-    if (err != cudaSuccess) return cuda_fail(err, "def_step_rows_apply kernel launch");
-    ctx->launches += 1;
+    if (side_stream && side_stream == (void *)ctx->stream)
+        return fail(DEF_ERR_ARG, "the side stream must differ from the context's stream");
+    if (side_stream && !ctx->rows_fork) {
+        int rc = check_device(ctx);
+        if (rc != DEF_OK) return rc;
+        cudaError_t err = cudaEventCreateWithFlags(&ctx->rows_fork, cudaEventDisableTiming);
+        if (err == cudaSuccess) err = cudaEventCreateWithFlags(&ctx->rows_join, cudaEventDisableTiming);
+        if (err != cudaSuccess) return cuda_fail(err, "creating the side stream's events");
+    }
+    ctx->rows_stream = (cudaStream_t)side_stream;
     return DEF_OK;
 }
 

@@ -115,7 +115,7 @@ struct StepArgs {
     float *m;            // [W, ld] or nullptr
     float *z;            // [W, ld] next detach points x_{t+1} - lambda e_{t+1}, or nullptr
     float *block_sum;    // [k] or nullptr: if set, the workers' sum of C(p) on block coordinate
-                         // (s + i) mod d goes to block_sum[i] and x is left alone (rows sharded
+                         // (s + i) mod d goes to block_sum[i] and x is only read (rows sharded
                          // over GPUs: the caller all-reduces block_sum, then applies it)
     int64_t n;           // local coordinates
     int64_t ld;          // row stride in floats
@@ -140,6 +140,25 @@ __device__ __forceinline__ int64_t cta_block_start(const StepArgs &a) {
     if (threadIdx.x == 0) s_shared = block_start(a.seed, a.step, a.d);
     __syncthreads();
     return s_shared;
+}
+
+// Programmatic dependent launch, used by the kernel pair of a step.  The kernel that does the tiles
+// touching the block (the primary) releases its dependents at its first instruction; the stream
+// kernel launched behind it (the secondary) may then start beside it -- the two write disjoint
+// floats.  What is enqueued AFTER the pair is ordered behind the secondary only, so the secondary
+// grid must not complete before the primary has: one thread of it (thread 0 of CTA 0) ends with
+// grid_dependency_wait(), which returns once the primary grid has completed and its writes are
+// visible, and a grid is complete only when all of its threads are.  One waiting thread is enough
+// for that and keeps one CTA slot busy; with the wait in every thread, finished CTAs would hold
+// their slots until the primary ends and the rest of the secondary could not start (measured:
+// +2 us on an 80 MB step).  The dependents are released only when every CTA of the primary has
+// started, so the wait cannot deadlock; in a kernel that was launched without the programmatic
+// attribute both instructions do nothing.
+__device__ __forceinline__ void release_dependent_grids() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void grid_dependency_wait() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 // One worker's row for V coordinates: Eq. 10 (or Algorithm 1's error-feedback step), then its new error.
@@ -236,8 +255,14 @@ __device__ __forceinline__ void column_group(const StepArgs &a, int64_t s, int64
 #pragma unroll
     for (int i = 0; i < V; ++i) {
         if (in[i]) {
-            x.v[i] = __fsub_rn(x.v[i], __fdiv_rn(sent[i], a.W_float));
-            a.x[col + i] = x.v[i];
+            if (a.block_sum) {                              // rows sharded over GPUs: x_{t+1} is not known yet on a
+                int64_t o = off + i;                        // block coordinate; z gets x_t there for now and the
+                if (o >= a.d) o -= a.d;                     // apply kernel overwrites it after the all-reduce
+                a.block_sum[o] = sent[i];
+            } else {
+                x.v[i] = __fsub_rn(x.v[i], __fdiv_rn(sent[i], a.W_float));
+                a.x[col + i] = x.v[i];
+            }
         }
     }
     float *zp = a.z + col;
@@ -273,8 +298,7 @@ def_step_kernel(const StepArgs a) {
 
 // Kernels for 16-byte aligned rows.  The n local coordinates are cut into tiles of
 // TILE = kTileThreads * 4 coordinates.  A tile "touches the block" if any of its coordinates
-// is one of the k block coordinates; every CTA decides that from the block start before it
-// issues a load.
+// is one of the k block coordinates; every CTA decides that from the block start.
 constexpr int kTileThreads = 256;
 constexpr int64_t kTile = (int64_t)kTileThreads * 4;
 
@@ -290,7 +314,7 @@ __device__ __forceinline__ bool tile_touches_block(const StepArgs &a, int64_t s,
 // sum: C(p) = 0 and e' = p.  The grid is (tiles, W) and CTA (t, w) does worker w's row of
 // tile t: three 16-byte loads and two stores per thread, few registers, full occupancy.
 // Consecutive CTAs sweep one row after the other, so the memory system sees a handful of
-// long sequential streams.  CTAs of tiles that touch the block leave at once.
+// long sequential streams.  CTAs of tiles that touch the block store nothing.
 // With DETACH the kernel also writes z_w = x - lambda e'_w for its row (x is unchanged outside
 // the block), which makes x a sixth stream that every worker's CTA of a tile reads.  ORDER
 // chooses how CTAs are numbered, i.e. what runs together:
@@ -306,7 +330,6 @@ constexpr int kOrderRows = 0, kOrderChunked = 1;
 template <bool MOM, int POL, bool DETACH = false, int ORDER = kOrderRows, int TILES = 1>
 __global__ void __launch_bounds__(kTileThreads * TILES)
 def_step_stream_kernel(const StepArgs a) {
-    const int64_t s = cta_block_start(a);
     int64_t first;
     unsigned w;
     if (ORDER == kOrderRows) {
@@ -320,24 +343,31 @@ def_step_stream_kernel(const StepArgs a) {
     }
     const int64_t tile = first * TILES + (int64_t)(threadIdx.x / kTileThreads);
     const int64_t col = tile * kTile + (int64_t)(threadIdx.x % kTileThreads) * 4;
-    if (col >= a.n || tile_touches_block(a, s, tile)) return;
+    const bool live = col < a.n;
     const size_t at = (size_t)w * (size_t)a.ld + (size_t)col;
-    const Vec<4> g = load_vec<4, POL>(a.g + at);
-    const Vec<4> e = load_vec<4, POL>(a.e + at);
-    Vec<4> m, m_new, e_new, x;
-    if (MOM) m = load_vec<4, POL>(a.m + at);
-    if (DETACH) x = load_vec<4, kCacheDefault>(a.x + col);
-    const bool none[4] = {false, false, false, false};
-    float unused[4];
-    worker_row<4, MOM>(g, m, e, none, a.eta, a.mu, true, m_new, e_new, unused);
-    if (MOM) store_vec<4, POL>(a.m + at, m_new);
-    store_vec<4, POL>(a.e + at, e_new);
-    if (DETACH) {
-        Vec<4> z;
+    // (Issuing the loads before the CTA learns the block start -- they do not depend on it -- was
+    // measured 2 % slower on the largest workload and no faster on the small ones.)
+    const int64_t s = cta_block_start(a);
+    if (live && !tile_touches_block(a, s, tile)) {
+        const Vec<4> g = load_vec<4, POL>(a.g + at);
+        const Vec<4> e = load_vec<4, POL>(a.e + at);
+        Vec<4> m, x;
+        if (MOM) m = load_vec<4, POL>(a.m + at);
+        if (DETACH) x = load_vec<4, kCacheDefault>(a.x + col);
+        Vec<4> m_new, e_new;
+        const bool none[4] = {false, false, false, false};
+        float unused[4];
+        worker_row<4, MOM>(g, m, e, none, a.eta, a.mu, true, m_new, e_new, unused);
+        if (MOM) store_vec<4, POL>(a.m + at, m_new);
+        store_vec<4, POL>(a.e + at, e_new);
+        if (DETACH) {
+            Vec<4> z;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) z.v[i] = __fmaf_rn(-a.lambda, e_new.v[i], x.v[i]);
-        store_vec<4, POL>(a.z + at, z);
+            for (int i = 0; i < 4; ++i) z.v[i] = __fmaf_rn(-a.lambda, e_new.v[i], x.v[i]);
+            store_vec<4, POL>(a.z + at, z);
+        }
     }
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) grid_dependency_wait();
 }
 
 // Tiles that touch the block: one CTA per tile walks the W rows in order (column_group).
@@ -352,7 +382,7 @@ def_step_block_kernel(const StepArgs a) {
     // The stream kernel that follows in the stream works on other tiles and needs nothing from
     // this kernel: when it was launched with programmatic stream serialization, let its CTAs
     // start now instead of after this grid has drained (a no-op otherwise).
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    release_dependent_grids();
     const int64_t s = cta_block_start(a);
     // the two runs in model coordinates, clipped to the local range [j0, j0 + n)
     const int64_t lo = a.j0, hi = a.j0 + a.n;
@@ -392,7 +422,7 @@ __global__ void __launch_bounds__(256)
 def_step_block_columns_kernel(const StepArgs a) {
     // the flat kernel that follows touches no float of a block coordinate: let it start now
     // when it was launched with programmatic stream serialization
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    release_dependent_grids();
     const int64_t s = cta_block_start(a);
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;   // i-th block coordinate
     if (i >= a.k) return;
@@ -402,52 +432,10 @@ def_step_block_columns_kernel(const StepArgs a) {
     if (col >= 0 && col < a.n) column_group<1, MOM, U, POL>(a, s, col);
 }
 
-template <bool MOM, int POL>
-__global__ void __launch_bounds__(kFlatThreads)
-def_step_flat_kernel(const StepArgs a) {
-    __shared__ int64_t shared[3];
-    const int64_t total = (int64_t)a.W * a.n;                 // rows are contiguous: ld == n
-    const int64_t base = (int64_t)blockIdx.x * kFlatTile;
-    if (threadIdx.x == 0) {
-        shared[0] = block_start(a.seed, a.step, a.d);
-        shared[1] = base / a.n;                               // worker of the CTA's first float
-        shared[2] = base - shared[1] * a.n;                   // and its coordinate
-    }
-    __syncthreads();
-    const int64_t s = shared[0];
-    const int64_t f = base + (int64_t)threadIdx.x * 4;
-    if (f >= total) return;
-    int64_t c = shared[2] + (int64_t)threadIdx.x * 4;        // < 2 n because n >= kFlatTile
-    if (c >= a.n) c -= a.n;
-    bool in[4];
-    bool any = false;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        int64_t ci = c + i;                                   // coordinate of float f + i (next row after a wrap)
-        if (ci >= a.n) ci -= a.n;
-        int64_t off = a.j0 + ci - s;
-        if (off < 0) off += a.d;
-        in[i] = off < a.k;
-        any |= in[i];
-    }
-    bool all = true;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) all &= in[i];
-    if (all) return;                                          // the block's floats belong to the other kernel
-    if (!any && f + 4 <= total) {
-        const bool none[4] = {false, false, false, false};
-        float unused[4];
-        const Vec<4> g = load_vec<4, POL>(a.g + f);
-        const Vec<4> e = load_vec<4, POL>(a.e + f);
-        Vec<4> m, m_new, e_new;
-        if (MOM) m = load_vec<4, POL>(a.m + f);
-        worker_row<4, MOM>(g, m, e, none, a.eta, a.mu, true, m_new, e_new, unused);
-        if (MOM) store_vec<4, POL>(a.m + f, m_new);
-        store_vec<4, POL>(a.e + f, e_new);
-        return;
-    }
-    // a group that straddles an edge of the block, or the last W * n % 4 floats: float by float,
-    // touching nothing that is in the block
+// The floats of one flat group of four, done one at a time: those that are not block coordinates
+// and lie inside the tensor.
+template <bool MOM>
+__device__ __forceinline__ void flat_group_by_floats(const StepArgs &a, int64_t f, int64_t total, const bool (&in)[4]) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         if (in[i] || f + i >= total) continue;
@@ -463,16 +451,71 @@ def_step_flat_kernel(const StepArgs a) {
     }
 }
 
+template <bool MOM, int POL>
+__global__ void __launch_bounds__(kFlatThreads)
+def_step_flat_kernel(const StepArgs a) {
+    __shared__ int64_t shared[3];
+    const int64_t total = (int64_t)a.W * a.n;                 // rows are contiguous: ld == n
+    const int64_t base = (int64_t)blockIdx.x * kFlatTile;
+    const int64_t f = base + (int64_t)threadIdx.x * 4;
+    const bool whole = f + 4 <= total;
+    if (threadIdx.x == 0) {
+        shared[0] = block_start(a.seed, a.step, a.d);
+        shared[1] = base / a.n;                               // worker of the CTA's first float
+        shared[2] = base - shared[1] * a.n;                   // and its coordinate
+    }
+    __syncthreads();
+    const int64_t s = shared[0];
+    if (f < total) {
+        int64_t c = shared[2] + (int64_t)threadIdx.x * 4;    // < 2 n because n >= kFlatTile
+        if (c >= a.n) c -= a.n;
+        bool in[4];
+        bool any = false, all = true;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            int64_t ci = c + i;                               // coordinate of float f + i (next row after a wrap)
+            if (ci >= a.n) ci -= a.n;
+            int64_t off = a.j0 + ci - s;
+            if (off < 0) off += a.d;
+            in[i] = off < a.k;
+            any |= in[i];
+            all &= in[i];
+        }
+        if (!any && whole) {
+            const bool none[4] = {false, false, false, false};
+            float unused[4];
+            const Vec<4> g = load_vec<4, POL>(a.g + f);
+            const Vec<4> e = load_vec<4, POL>(a.e + f);
+            Vec<4> m, m_new, e_new;
+            if (MOM) m = load_vec<4, POL>(a.m + f);
+            worker_row<4, MOM>(g, m, e, none, a.eta, a.mu, true, m_new, e_new, unused);
+            if (MOM) store_vec<4, POL>(a.m + f, m_new);
+            store_vec<4, POL>(a.e + f, e_new);
+        } else if (!all) {
+            // a group that straddles an edge of the block, or the last W * n % 4 floats: float by
+            // float, touching nothing that is in the block (whose floats belong to the other kernel)
+            flat_group_by_floats<MOM>(a, f, total, in);
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) grid_dependency_wait();
+}
+
 // Second half of a row-sharded step (Algorithm 1's update after the all-reduce):
-// x[(s + i) mod d] -= block_sum[i] / W_total for the k block coordinates.
+// x[(s + i) mod d] -= block_sum[i] / W_total for the k block coordinates.  With z set it also
+// writes the next detach point of the W_local local workers there: e' = +0 on a block
+// coordinate, so z[w, j] = x_{t+1}[j] for every w.
 __global__ void __launch_bounds__(256)
-def_apply_block_kernel(float *__restrict__ x, const float *__restrict__ block_sum, StepArgs a) {
+def_apply_block_kernel(float *__restrict__ x, const float *__restrict__ block_sum, float *__restrict__ z,
+                       int W_local, StepArgs a) {
     const int64_t s = cta_block_start(a);
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= a.k) return;
     int64_t j = s + i;
     if (j >= a.d) j -= a.d;
-    x[j] = __fsub_rn(x[j], __fdiv_rn(block_sum[i], a.W_float));
+    const float x_new = __fsub_rn(x[j], __fdiv_rn(block_sum[i], a.W_float));
+    x[j] = x_new;
+    if (z)
+        for (int w = 0; w < W_local; ++w) z[(size_t)w * (size_t)a.ld + (size_t)j] = x_new;
 }
 
 }  // namespace defk

@@ -9,13 +9,18 @@ of synthetic gradients.  The timed workload is the VGG-16-sized one (d = 138,357
 W = 16, k = d/32, DEF, momentum 0.9): its 35 GB of state and gradients are far larger
 than the L2, so no flush is needed between iterations.  Prints ONE JSON line on rank 0.
 
-With N > 1 (launched by torch.distributed.run) every rank holds a d-column shard of an
-N*d-dimensional model (def_step_columns): the step is separate per coordinate, so the
-shards need no exchange, per-GPU work is fixed ("weak" scaling), and the value is the
-elements all ranks processed divided by the slowest rank's device time.
+With N > 1 (launched by torch.distributed.run) the WORKERS are cut across the ranks, as in the
+paper's own deployment: every rank holds W = 16 workers' rows of the full d-dimensional model and
+a replica of x, so there are K = 16 N workers; a step is the local half (momentum, error feedback,
+new error, the local workers' block sums), one NCCL all-reduce of the k block sums -- issued on a
+side stream so that it overlaps the streaming kernel -- and the update.  Per-GPU work is fixed
+("weak" scaling); the value is the elements all ranks processed divided by the slowest rank's
+device time.  --sharding columns gives every rank a d-column shard of an N*d-dimensional model
+instead (no exchange at all: the step is separate per coordinate).
 
---impl reference times the CPU oracle (plain C, single thread) on a bounded sample of the
-same workload; it is a deliberately slow program, reported as a baseline only.
+--impl reference times the CPU oracle (plain C; the same source built with OpenMP for all host
+cores, and the single-threaded build beside it) on a bounded sample of the same workload; it is a
+deliberately slow program, reported as a baseline only.
 """
 import argparse
 import hashlib

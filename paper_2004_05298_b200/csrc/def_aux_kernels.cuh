@@ -135,12 +135,15 @@ def_stats_partial_kernel(const float *__restrict__ e, int64_t n, int64_t ld, int
                     }
             }
         } else {                                // the n % V coordinates at the end
-            for (int64_t c = col; c < n; ++c)
+#pragma unroll
+            for (int i = 0; i < V; ++i) {       // (i is a compile-time index: s1 stays in registers)
+                if (col + i >= n) continue;
                 for (int w = 0; w < W; ++w) {
-                    const double v = (double)e[(size_t)w * (size_t)ld + (size_t)c];
-                    s1[c - col] += v;
+                    const double v = (double)e[(size_t)w * (size_t)ld + (size_t)(col + i)];
+                    s1[i] += v;
                     sq = fma(v, v, sq);
                 }
+            }
         }
 #pragma unroll
         for (int i = 0; i < V; ++i) {

@@ -10,3 +10,8 @@ extern "C" void aten_philox4x32_10(uint64_t seed, uint64_t subsequence, uint64_t
   at::Philox4_32 engine(seed, subsequence, offset);
   for (int i = 0; i < 4; ++i) out[i] = engine();
 }
+
+extern "C" void aten_philox4x32_10_batch(int64_t n, const uint64_t *seeds, const uint64_t *subsequences,
+                                         const uint64_t *offsets, uint32_t *out) {
+  for (int64_t i = 0; i < n; ++i) aten_philox4x32_10(seeds[i], subsequences[i], offsets[i], out + 4 * i);
+}

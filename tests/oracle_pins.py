@@ -379,6 +379,8 @@ def aten_philox():
         lib = ctypes.CDLL(out)
         lib.aten_philox4x32_10.argtypes = [ctypes.c_uint64] * 3 + [ctypes.c_void_p]
         lib.aten_philox4x32_10.restype = None
+        lib.aten_philox4x32_10_batch.argtypes = [ctypes.c_int64] + [ctypes.c_void_p] * 4
+        lib.aten_philox4x32_10_batch.restype = None
         _aten = lib
     return _aten
 
@@ -403,6 +405,42 @@ def pin_philox_against_library_engine(o):
     # fewer rounds are a different bijection (guards the round count)
     assert o.philox4x32((1, 2, 3, 4), (5, 6), 7) == philox4x32_bigint((1, 2, 3, 4), (5, 6), 7)
     assert o.philox4x32((1, 2, 3, 4), (5, 6), 7) != o.philox4x32((1, 2, 3, 4), (5, 6), 10)
+
+
+def philox4x32_numpy(ctr, key, rounds=10):
+    """The same bijection on whole arrays: ctr [n, 4] and key [n, 2] as uint64 holding 32-bit words."""
+    c0, c1, c2, c3 = (ctr[:, i].astype(np.uint64) for i in range(4))
+    k0, k1 = key[:, 0].astype(np.uint64), key[:, 1].astype(np.uint64)
+    mask, sh = np.uint64(_M32), np.uint64(32)
+    for _ in range(rounds):
+        p0 = np.uint64(0xD2511F53) * c0
+        p1 = np.uint64(0xCD9E8D57) * c2
+        c0, c1, c2, c3 = (p1 >> sh) ^ c1 ^ k0, p1 & mask, (p0 >> sh) ^ c3 ^ k1, p0 & mask
+        k0, k1 = (k0 + np.uint64(0x9E3779B9)) & mask, (k1 + np.uint64(0xBB67AE85)) & mask
+    return np.stack([c0, c1, c2, c3], axis=1).astype(np.uint32)
+
+
+def pin_philox_million_pairs(o):
+    """2^20 random (counter, key) pairs: the oracle's generator against the library engine and
+    against the array statement above, word for word."""
+    n = 1 << 20
+    rng = _rng(53)
+    seeds = rng.integers(0, 2 ** 64, size=n, dtype=np.uint64)
+    subs = rng.integers(0, 2 ** 64, size=n, dtype=np.uint64)
+    offs = rng.integers(0, 2 ** 64, size=n, dtype=np.uint64)
+    seeds[: n // 4] %= 8; offs[: n // 4] %= 100000; subs[: n // 4] = 0x52424753   # what the steps really draw from
+    lo, hi = (lambda v: v & np.uint64(_M32)), (lambda v: v >> np.uint64(32))
+    ctr = np.ascontiguousarray(np.stack([lo(offs), hi(offs), lo(subs), hi(subs)], axis=1).astype(np.uint32))
+    key = np.ascontiguousarray(np.stack([lo(seeds), hi(seeds)], axis=1).astype(np.uint32))
+    got = np.empty((n, 4), np.uint32)
+    f = o.lib.def_oracle_philox4x32
+    c0, k0, g0 = ctr.ctypes.data, key.ctypes.data, got.ctypes.data
+    for i in range(n):
+        f(c0 + 16 * i, k0 + 8 * i, 10, g0 + 16 * i)
+    want = np.empty((n, 4), np.uint32)
+    aten_philox().aten_philox4x32_10_batch(n, seeds.ctypes.data, subs.ctypes.data, offs.ctypes.data, want.ctypes.data)
+    assert np.array_equal(got, want)
+    assert np.array_equal(got, philox4x32_numpy(ctr, key))
 
 
 def pin_block_start(o):
@@ -472,6 +510,7 @@ ALL_PINS = [
     ("f32_tracks_f64", pin_f32_tracks_f64),
     ("column_view", pin_column_view),
     ("philox_against_library_engine", pin_philox_against_library_engine),
+    ("philox_million_pairs", pin_philox_million_pairs),
     ("block_start", pin_block_start),
     ("distances", pin_distances),
 ]

@@ -12,6 +12,8 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
+
 pytestmark = pytest.mark.gpu
 
 STATS_TOL = 2e-9      # of stats[0]; the tolerance tests/test_aux_gpu.py uses for the distances
@@ -52,16 +54,26 @@ def test_two_calls_in_a_row_match_def_stats(B):
     big = _errors(8, 3_000_000, seed=1)
     small = _errors(3, 70_001, seed=2, offset=1)            # odd n, 4-byte aligned rows
     out = torch.full((3,), -1.0, dtype=torch.float64, device="cuda")
-    before = torch.cuda.memory_allocated()
+    host = torch.empty(3, dtype=torch.float64).pin_memory()
+    B.def_stats_static(small, lam, out)                     # the one-time address look-up, if this process has not done it
+    torch.cuda.synchronize()
+    # From here on the device's free memory must not move: cudaMemGetInfo sees every allocation
+    # of the process, the library's own included (torch's counters would only see torch's pool).
+    pool_before = torch.cuda.memory_allocated()
+    free_before = torch.cuda.mem_get_info()[0]
     results = []
     for e in (big, small, big):
         B.def_stats_static(e, lam, out)
+        host.copy_(out, non_blocking=True)                  # into pinned memory allocated above: no new buffer
         torch.cuda.synchronize()
-        results.append(out.cpu().numpy().copy())
-    assert torch.cuda.memory_allocated() == before          # nothing was taken from torch's pool either
+        results.append(host.numpy().copy())
+        assert torch.cuda.mem_get_info()[0] >= free_before, "device memory was allocated during the call"
+    assert torch.cuda.memory_allocated() == pool_before     # nothing was taken from torch's pool either
     for e, got in zip((big, small, big), results):
-        want = _reference(B, e, lam)
+        want = _reference(B, e, lam)                        # the existing entry point
         assert np.all(np.abs(got - want) <= STATS_TOL * want[0]), (got, want)
+        truth = np.array(oracle.stats(e.cpu().numpy(), lam))   # and the CPU oracle's plain loops
+        assert np.all(np.abs(got - truth) <= STATS_TOL * truth[0]), (got, truth)
     assert np.array_equal(results[0], results[2]), "same input, same bits, whatever ran in between"
 
 

@@ -156,9 +156,11 @@ def _max_over_ranks(dist, value):
 
 
 def time_steps(B, ctx, shard, tensors, steps, warmup, seed, dist=None, flush=None, sample_clocks=None, step_fn=None):
-    """Device time of `steps` steps.  Without `flush`: one event pair around the whole loop,
-    launches back to back.  With `flush` (a buffer larger than the L2 that is rewritten
-    between iterations): one event pair per step, summed."""
+    """Device time of `steps` steps, from CUDA events on the stream the steps are enqueued on.
+    Without `flush`: an event before the first step and one after every step, launches back to
+    back (the total is first event to last).  With `flush` (a buffer larger than the L2 that is
+    rewritten between iterations): one event pair per step, summed.  Returns (total ms, max over
+    ranks; launches; this rank's per-step ms)."""
     import torch
     j0, n, ld = shard
     x, g, e, m = tensors
@@ -172,13 +174,14 @@ def time_steps(B, ctx, shard, tensors, steps, warmup, seed, dist=None, flush=Non
     if sample_clocks is not None:
         sample_clocks.start()
     if flush is None:
-        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        start.record()
+        marks = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        marks[0].record()
         for t in range(steps):
             step_fn(warmup + t)
-        end.record()
+            marks[t + 1].record()
         torch.cuda.synchronize()
-        ms = start.elapsed_time(end)
+        ms = marks[0].elapsed_time(marks[-1])
+        per_step = [marks[t].elapsed_time(marks[t + 1]) for t in range(steps)]
     else:
         pairs = []
         for t in range(steps):
@@ -189,10 +192,16 @@ def time_steps(B, ctx, shard, tensors, steps, warmup, seed, dist=None, flush=Non
             b.record()
             pairs.append((a, b))
         torch.cuda.synchronize()
-        ms = sum(a.elapsed_time(b) for a, b in pairs)
+        per_step = [a.elapsed_time(b) for a, b in pairs]
+        ms = sum(per_step)
     _barrier(dist)
     launches = B.def_launch_count(ctx) - launches0
-    return _max_over_ranks(dist, ms), launches
+    return _max_over_ranks(dist, ms), launches, per_step
+
+
+def step_spread(per_step):
+    """Median and minimum of the per-step device times (this rank's)."""
+    return {"ms_per_step_median": statistics.median(per_step), "ms_per_step_min": min(per_step)}
 
 
 TILE = 1024   # coordinates per tile of the two step kernels (256 threads x 4)
@@ -211,12 +220,16 @@ def touched_columns(d, k, s, j0, n):
     return sum(min(TILE, n - t * TILE) for t in tiles)
 
 
-def profile_kernels(B, ctx, shard, tensors, steps, first_step, seed, per_el, k_share, flush=None):
+def profile_kernels(B, ctx, shard, tensors, steps, first_step, seed, per_el, k_share, flush=None, step_fn=None):
     """Per-kernel device time over `steps` more steps (each launch bracketed by events inside the
-    library and waited for), with the algorithmic bytes each kernel had to move."""
+    library, on the stream it is launched on, and waited for), with the algorithmic bytes each
+    kernel had to move."""
     j0, n, ld = shard
     x, g, e, m = tensors
     W = ctx.W
+    if step_fn is None:
+        def step_fn(t):
+            B.def_step_columns(ctx, j0, n, ld, x, g, e, m, t, seed)
     before = {kind: B.def_kernel_time(ctx, kind) for kind in (B.DEF_KERNEL_STREAM, B.DEF_KERNEL_BLOCK, B.DEF_KERNEL_GENERAL)}
     B.def_set_kernel_timing(ctx, True)
     bytes_stream = bytes_block = bytes_general = 0
@@ -224,7 +237,7 @@ def profile_kernels(B, ctx, shard, tensors, steps, first_step, seed, per_el, k_s
         if flush is not None:
             flush.add_(1.0)
         step = first_step + t
-        B.def_step_columns(ctx, j0, n, ld, x, g, e, m, step, seed)
+        step_fn(step)
         cols = touched_columns(ctx.d, ctx.k, B.def_block_start(ctx, step, seed), j0, n)
         bytes_block += per_el * W * cols + 8 * k_share
         bytes_stream += per_el * W * (n - cols)
@@ -243,30 +256,91 @@ def profile_kernels(B, ctx, shard, tensors, steps, first_step, seed, per_el, k_s
     return out
 
 
-def bench_rows(B, WL, wl, steps, warmup, dist, world, rank, sampler=None):
+def bench_rows(B, WL, wl, steps, warmup, dist, world, rank, sampler=None, side_stream=True, detach=False,
+               profile=False):
     """Workers cut across ranks (the paper's deployment): every rank holds W rows of the full model and
-    a replica of x; one step = local half, NCCL all-reduce of the k block sums, apply."""
+    a replica of x; one step = local half, NCCL all-reduce of the k block sums (on a side stream,
+    beside the streaming kernel, unless side_stream is off), apply.  With `detach` the step also
+    writes the local workers' next detach points (24 instead of 20 bytes per gradient element)."""
     import torch
     dev = torch.device("cuda")
     ctx = B.def_create(wl.d, wl.W, wl.k, wl.variant, wl.lr, wl.momentum, (wl.lam, 0.0))
+    side = torch.cuda.Stream() if side_stream else None
+    if side is not None:
+        B.def_set_rows_stream(ctx, side)
     x = WL.initial_params(wl, dev)
     e, m = WL.zeros_state(wl, dev)
     g = WL.gradients(wl, rank, dev)
+    z = torch.empty(wl.W, wl.d, dtype=torch.float32, device=dev) if detach else None
     block = torch.zeros(wl.k, dtype=torch.float32, device=dev)
 
     def step_fn(t):
-        B.def_step_rows(ctx, x, g, e, m, block, t, wl.rbgs_seed)
+        B.def_step_rows(ctx, x, g, e, m, block, t, wl.rbgs_seed, detached_out=z)
 
-    ms, launches = time_steps(B, ctx, (0, wl.d, wl.d), (x, g, e, m), steps, warmup, wl.rbgs_seed, dist, None, sampler, step_fn)
+    ms, launches, per_step = time_steps(B, ctx, (0, wl.d, wl.d), (x, g, e, m), steps, warmup, wl.rbgs_seed, dist, None,
+                                        sampler, step_fn)
+    per_el = 24 if detach else 20
+    # local rows, the k block sums written, read and applied to x, and (detach) x read once
+    alg_bytes = per_el * wl.W * wl.d + 16 * wl.k + (4 * wl.d if detach else 0)
+    kernels = None
+    if profile:
+        kernels = profile_kernels(B, ctx, (0, wl.d, wl.d), (x, g, e, m), min(steps, 5), warmup + steps, wl.rbgs_seed,
+                                  per_el, 0.5 * wl.k, None, step_fn)
+    if side is not None:
+        B.def_set_rows_stream(ctx, None)
+    B.def_destroy(ctx)
+    del x, g, e, m, z
+    torch.cuda.empty_cache()
+    return ms, launches, world * wl.W * wl.d, alg_bytes, kernels, per_step
+
+
+def bench_rows_e2e(B, WL, wl, steps, warmup, dist, world, rank):
+    """The row-sharded step with the step's input in host memory: every step copies the local
+    workers' gradients [W, d] in from pinned host memory, runs def_step_rows, and copies the k
+    updated block coordinates' sums out (what a training loop would log or checkpoint)."""
+    import torch
+    dev = torch.device("cuda")
+    ctx = B.def_create(wl.d, wl.W, wl.k, wl.variant, wl.lr, wl.momentum, (wl.lam, 0.0))
+    side = torch.cuda.Stream()
+    B.def_set_rows_stream(ctx, side)
+    x = WL.initial_params(wl, dev)
+    e, m = WL.zeros_state(wl, dev)
+    g = WL.gradients(wl, rank, dev)
+    g_host = torch.empty(wl.W, wl.d, dtype=torch.float32, pin_memory=True)
+    g_host.copy_(g)
+    block = torch.zeros(wl.k, dtype=torch.float32, device=dev)
+    block_host = torch.empty(wl.k, dtype=torch.float32, pin_memory=True)
+
+    def step_fn(t):
+        g.copy_(g_host, non_blocking=True)
+        B.def_step_rows(ctx, x, g, e, m, block, t, wl.rbgs_seed)
+        block_host.copy_(block, non_blocking=True)
+
+    for t in range(warmup):
+        step_fn(t)
+    _barrier(dist)
+    t0 = time.perf_counter()
+    for t in range(steps):
+        step_fn(warmup + t)
+    torch.cuda.synchronize()
+    sec = time.perf_counter() - t0
+    _barrier(dist)
+    sec = _max_over_ranks(dist, sec)
+    B.def_set_rows_stream(ctx, None)
     B.def_destroy(ctx)
     del x, g, e, m
     torch.cuda.empty_cache()
-    return ms, launches, world * wl.W * wl.d, 20 * wl.W * wl.d + 12 * wl.k
+    return {"value": world * wl.W * wl.d * steps / sec, "unit": UNIT,
+            "h2d_bytes_per_step": 4 * wl.W * wl.d, "d2h_bytes_per_step": 4 * wl.k,
+            "steps": steps, "ms_per_step": 1e3 * sec / steps,
+            "api": "binding.def_step_rows; gradients copied in from pinned host memory and the k block sums copied "
+                   "out every step (errors, momentum and the model stay on the GPU)"}
 
 
 def bench_workload(B, WL, wl, steps, warmup, dist, world, rank, sampler=None, flush=None, profile=False):
-    """Allocate a rank's shard of the workload, run, return (ms, launches, elements per step over
-    all ranks, algorithmic bytes per step on this rank, per-kernel profile or None)."""
+    """Allocate a rank's column shard of the workload (the whole model on one rank), run, return
+    (ms, launches, elements per step over all ranks, algorithmic bytes per step on this rank,
+    per-kernel profile or None, this rank's per-step ms)."""
     import torch
     dev = torch.device("cuda")
     d_global = wl.d * world
@@ -279,7 +353,7 @@ def bench_workload(B, WL, wl, steps, warmup, dist, world, rank, sampler=None, fl
         m = None
     col_sigma = WL.column_sigma(wl, dev) if wl.grad == "per_tensor" else None
     g = WL.gradients(wl, rank, dev, col_sigma=col_sigma)   # one gradient buffer, reused: values do not steer the kernel
-    ms, launches = time_steps(B, ctx, (j0, n, n), (x, g, e, m), steps, warmup, wl.rbgs_seed, dist, flush, sampler)
+    ms, launches, per_step = time_steps(B, ctx, (j0, n, n), (x, g, e, m), steps, warmup, wl.rbgs_seed, dist, flush, sampler)
     per_el = 20 if wl.momentum != 0.0 else 12
     alg_bytes = per_el * wl.W * n + 8 * k_global / world
     kernels = None
@@ -289,7 +363,7 @@ def bench_workload(B, WL, wl, steps, warmup, dist, world, rank, sampler=None, fl
     B.def_destroy(ctx)
     del x, g, e, m
     torch.cuda.empty_cache()
-    return ms, launches, wl.W * d_global, alg_bytes, kernels
+    return ms, launches, wl.W * d_global, alg_bytes, kernels, per_step
 
 
 def bench_aux(B, WL, wl, reps=5):
@@ -425,35 +499,48 @@ def bench_e2e(B, WL, wl, steps, warmup, dist, world, rank):
     return out
 
 
-def oracle_sample_run(WL, wl, steps, warmup, budget_s):
-    """Times the CPU oracle (as it stands, one thread) on a leading column range of the workload,
-    sized from a short probe so that warmup + steps stay within budget_s."""
+ORACLE_SAMPLE_COLUMNS = 8_000_000     # leading columns of the workload both CPU legs step over
+
+
+def oracle_time(o, wl, steps, warmup, n):
+    """Times one build of the CPU oracle (as it stands) on columns [0, n) of the workload, all W
+    workers: `warmup` untimed steps (they also fault the pages in), then `steps` timed ones.
+    Returns (elements/s, seconds, threads used)."""
     import numpy as np
-    import oracle
     rng = np.random.default_rng(0)
     d, W, k = wl.d, wl.W, wl.k
+    n = int(min(n, d))
+    g = ((wl.sigma or 0.01) * rng.standard_normal((W, n), dtype=np.float32)).astype(np.float32)
+    x, e, m = np.zeros(n, np.float32), np.zeros((W, n), np.float32), np.zeros((W, n), np.float32)
+    cols = None if n == d else np.arange(n, dtype=np.int64)
 
-    def make(n):
-        g = (wl.sigma or 0.01) * rng.standard_normal((W, n), dtype=np.float32)
-        return (np.zeros(n, np.float32), g, np.zeros((W, n), np.float32), np.zeros((W, n), np.float32),
-                np.arange(n, dtype=np.int64))
+    def run(t):
+        o.step(x, g, e, m, d=d, k=k, s=o.block_start(wl.rbgs_seed, t, d), eta=wl.lr, mu=wl.momentum, cols=cols)
 
-    def run(state, t):
-        x, g, e, m, cols = state
-        s = oracle.block_start(wl.rbgs_seed, t, d)
-        oracle.step(x, g, e, m, d=d, k=k, s=s, eta=wl.lr, mu=wl.momentum, cols=cols if len(cols) != d else None)
-
-    probe = make(min(d, 250_000))
-    t0 = time.perf_counter(); run(probe, 0); rate = W * len(probe[4]) / (time.perf_counter() - t0)
-    n = int(min(d, max(1000, rate * budget_s / (steps + warmup) / W)))
-    state = make(n)
     for t in range(warmup):
-        run(state, t)
+        run(t)
     t0 = time.perf_counter()
     for t in range(steps):
-        run(state, warmup + t)
+        run(warmup + t)
     sec = time.perf_counter() - t0
-    return W * n * steps / sec, sec, n
+    return W * n * steps / sec, sec, o.threads()
+
+
+def cpu_baseline(wl, steps_all, warmup_all, steps_one=8, warmup_one=1, n=ORACLE_SAMPLE_COLUMNS):
+    """The oracle on the host cores, both builds of the one source on the same sample with the
+    same protocol: OpenMP over the coordinate loops (all cores; the headline figure) and the
+    plain single-threaded build."""
+    import oracle
+    n = int(min(n, wl.d))
+    v_all, sec_all, cores = oracle_time(oracle.all_cores(), wl, steps_all, warmup_all, n)
+    v_one, sec_one, one = oracle_time(oracle.default(), wl, steps_one, warmup_one, n)
+    sample = ("each step = one oracle step on columns [0, %d) of d = %d, all W = %d workers; %d warm-up + %d timed "
+              "steps on %d threads (%.1f s), %d + %d on 1 thread (%.1f s)"
+              % (n, wl.d, wl.W, warmup_all, steps_all, cores, sec_all, warmup_one, steps_one, sec_one))
+    return {"value": v_all, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
+            "seconds": sec_all, "steps": steps_all,
+            "one_core": {"value": v_one, "unit": UNIT, "cores": one, "seconds": sec_one, "steps": steps_one},
+            "host_cores": os.cpu_count()}
 
 
 def run_reference(args):
@@ -461,29 +548,57 @@ def run_reference(args):
     if int(os.environ.get("RANK", "0")) != 0:
         return
     from paper_2004_05298_b200 import workloads as WL
-    wl = WL.get(5)
-    value, sec, n = oracle_sample_run(WL, wl, args.steps, args.warmup, budget_s=args.reference_budget_s)
-    sample = "each step = one oracle step on columns [0, %d) of d = %d, all W = %d workers" % (n, wl.d, wl.W)
+    wl = WL.get(args.cfg)
+    base = cpu_baseline(wl, args.steps, args.warmup, n=args.reference_columns)
     line = {
-        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sec / args.steps,
+        "impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * base["seconds"] / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": workload_config(wl, 1),
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
-        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "config": workload_config(wl, 1, "single"),
+        "cpu_baseline": base,
+        "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line))
 
 
-def workload_config(wl, world):
+def workload_config(wl, world, sharding):
     from paper_2004_05298_b200 import workloads as WL
-    return {"workload": "cfg%d %s: d=%d per GPU, W=%d, k=d/%d, %s, momentum %.1f, lr %.2f, fp32"
-                        % (wl.cfg, wl.name, wl.d, wl.W, wl.ratio, WL.VARIANT_NAMES[wl.variant], wl.momentum, wl.lr),
-            "d": wl.d * world, "W": wl.W, "k": max(1, wl.d * world // wl.ratio), "variant": WL.VARIANT_NAMES[wl.variant],
-            "parallelism": "columns sharded over %d GPU(s), no collective" % world,
-            "l2": ("inputs larger than L2 (%.1f GB per GPU); no flush" % (wl.algorithmic_bytes_per_step() * 0.8 / 1e9))
-            if wl.algorithmic_bytes_per_step() >= 1e9 else "L2 flushed between steps (384 MB buffer rewritten)"}
+    big = wl.algorithmic_bytes_per_step() >= 1e9
+    cfg = {"workload": "cfg%d %s: d=%d per GPU, W=%d per GPU, k=d/%d, %s, momentum %.1f, lr %.2f, fp32"
+                       % (wl.cfg, wl.name, wl.d, wl.W, wl.ratio, WL.VARIANT_NAMES[wl.variant], wl.momentum, wl.lr),
+           "variant": WL.VARIANT_NAMES[wl.variant],
+           "l2": ("inputs larger than L2 (%.1f GB per GPU); no flush" % (wl.algorithmic_bytes_per_step() * 0.8 / 1e9))
+           if big else "L2 flushed between steps (384 MB buffer rewritten)"}
+    if sharding == "rows":
+        cfg.update({"d": wl.d, "W": wl.W * world, "k": wl.k,
+                    "parallelism": "workers (rows) sharded over %d GPU(s): W = %d per GPU, K = %d workers in all, NCCL "
+                                   "all-reduce of the k = %d block sums per step on a side stream" % (world, wl.W, wl.W * world, wl.k)})
+    elif sharding == "columns":
+        cfg.update({"d": wl.d * world, "W": wl.W, "k": max(1, wl.d * world // wl.ratio),
+                    "parallelism": "columns sharded over %d GPU(s), no collective" % world})
+    else:
+        cfg.update({"d": wl.d, "W": wl.W, "k": wl.k, "parallelism": "one GPU holds all W workers (no collective)"})
+    return cfg
+
+
+def roofline_of(kernels, step_gbs, alg_bytes, launches_per_step, peak, peak_kind):
+    """The roofline object of the JSON line: the dominant kernel against the measured HBM peak."""
+    top = max(kernels, key=lambda kk: kk["ms_per_launch"] * kk["launches"])
+    achieved = top["GB/s"] if top["GB/s"] is not None else step_gbs
+    traffic = None
+    if (NCU_TRAFFIC_BYTES_PER_ELEMENT is not None and NCU_TRAFFIC_KERNEL_SHA256 == _kernel_hash()
+            and top["algorithmic_bytes_per_launch"] and top["kernel"] == "def_step_stream_kernel"):
+        traffic = NCU_TRAFFIC_BYTES_PER_ELEMENT * top["algorithmic_bytes_per_launch"] / 20.0
+    return {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+            "traffic": traffic, "peak_kind": "of %s" % peak_kind, "frac_of_8000_nominal": achieved / 8000.0,
+            "kernel": top["kernel"], "algorithmic_bytes_per_launch": top["algorithmic_bytes_per_launch"],
+            "launch_ms": top["ms_per_launch"],
+            "whole_step": {"GB/s": step_gbs, "frac": step_gbs / peak, "frac_of_8000_nominal": step_gbs / 8000.0,
+                           "algorithmic_bytes_per_step": alg_bytes, "launches_per_step": launches_per_step},
+            "kernels": kernels,
+            "note": "per-kernel times from a second pass of the same steps with each launch bracketed by "
+                    "CUDA events on the launching stream; whole_step is the timed region itself"}
 
 
 def main():
@@ -494,11 +609,14 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cfg", type=int, default=5, choices=[1, 2, 3, 4, 5],
                     help="workload to time (default 5, the largest; smaller ones are for profiling)")
-    ap.add_argument("--sharding", default="columns", choices=["columns", "rows"],
-                    help="columns (default): each rank holds a column range of every tensor, no collective; "
-                         "rows: each rank holds W workers of the full model and the k block sums are all-reduced (NCCL)")
-    ap.add_argument("--reference-budget-s", type=float, default=90.0,
-                    help="--impl reference: CPU seconds the whole run (warm-up + steps) may take")
+    ap.add_argument("--sharding", default="auto", choices=["auto", "single", "rows", "columns"],
+                    help="auto (default): one GPU runs def_step on all W workers; N > 1 GPUs cut the workers (rows) across "
+                         "ranks and all-reduce the k block sums (NCCL).  rows: that path, also on one GPU (a one-rank NCCL "
+                         "group).  columns: each rank holds a column range of every tensor, no collective")
+    ap.add_argument("--reference-columns", type=int, default=ORACLE_SAMPLE_COLUMNS,
+                    help="--impl reference: leading columns of the workload every oracle step runs over")
+    ap.add_argument("--no-side-stream", action="store_true",
+                    help="rows: keep the all-reduce and the update on the context's stream, behind the streaming kernel")
     ap.add_argument("--aux", action="store_true",
                     help="with --no-extras: still time the helpers (detach, output, stats, step with fused detach)")
     ap.add_argument("--no-extras", action="store_true",
@@ -517,61 +635,62 @@ def main():
     from paper_2004_05298_b200 import workloads as WL
 
     dist, world, rank, local = _dist_setup(args.gpus)
+    sharding = args.sharding
+    if sharding == "auto":
+        sharding = "single" if world == 1 else "rows"
+    if sharding == "single" and world > 1:
+        raise SystemExit("--sharding single needs one GPU")
+    if sharding == "columns" and world == 1:
+        sharding = "single"
     wl = WL.get(args.cfg)
-    if args.sharding == "rows":
+    peak, peak_kind = _measured_peak()
+    sampler = ClockSampler(local)
+    line = {"metric": METRIC, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": workload_config(wl, world, sharding)}
+
+    if sharding == "rows":
         import torch.distributed as tdist
-        if dist is None:                                   # one rank: still a real NCCL group
+        own_group = dist is None
+        if own_group:                                      # one rank: still a real NCCL group
             tdist.init_process_group("nccl", init_method="tcp://127.0.0.1:29581", rank=0, world_size=1,
                                      device_id=torch.device("cuda", 0))
-        sampler = ClockSampler(local)
-        ms, launches, elements, alg_bytes = bench_rows(B, WL, wl, args.steps, args.warmup, dist, world, rank, sampler)
+        side = not args.no_side_stream
+        if not side:
+            line["config"]["parallelism"] = line["config"]["parallelism"].replace("on a side stream", "on the step's own stream")
+        ms, launches, elements, alg_bytes, kernels, per_step = bench_rows(B, WL, wl, args.steps, args.warmup, dist, world, rank,
+                                                                          sampler, side_stream=side, profile=True)
         clocks = sampler.finish()
-        peak, peak_kind = _measured_peak()
-        gbs = alg_bytes * args.steps / (ms * 1e-3) / 1e9
-        cfg = workload_config(wl, world)
-        cfg["parallelism"] = "workers (rows) sharded over %d GPU(s): W = %d per GPU, NCCL all-reduce of k = %d floats per step" % (world, wl.W, wl.k)
-        cfg["d"], cfg["W"], cfg["k"] = wl.d, wl.W * world, wl.k
+        step_gbs = alg_bytes * args.steps / (ms * 1e-3) / 1e9
+        line.update({"value": elements * args.steps / (ms * 1e-3), "ms_per_step": ms / args.steps, **step_spread(per_step),
+                     "gpu_launches": launches, "clocks": clocks,
+                     "roofline": roofline_of(kernels, step_gbs, alg_bytes, launches / args.steps, peak, peak_kind)})
+        if args.aux or not args.no_extras:
+            ms_z, _, _, bytes_z, _, per_z = bench_rows(B, WL, wl, min(args.steps, 10), 3, dist, world, rank, None,
+                                                       side_stream=side, detach=True)
+            n_z = min(args.steps, 10)
+            line["aux"] = [{"op": "def_step_rows with the fused detach output", "ms": ms_z / n_z, "algorithmic_bytes": bytes_z,
+                            "GB/s": bytes_z * n_z / (ms_z * 1e-3) / 1e9, **step_spread(per_z)}]
+        if not args.no_extras:
+            line["e2e"] = bench_rows_e2e(B, WL, wl, max(1, min(args.steps, 3)), 1, dist, world, rank)
+            if world == 1:
+                line["cpu_baseline"] = cpu_baseline(wl, 20, 1)
         if rank == 0:
-            print(json.dumps({
-                "metric": METRIC, "value": elements * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
-                "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
-                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": cfg,
-                "gpu_launches": launches, "clocks": clocks,
-                "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
-                             "traffic": None, "peak_kind": "of %s" % peak_kind, "kernel": "whole step (local half + all-reduce + apply)"}}))
-        tdist.destroy_process_group()
+            print(json.dumps(line))
+        if own_group or dist is not None:
+            tdist.destroy_process_group()
         return
-    sampler = ClockSampler(local)
+
     small = wl.algorithmic_bytes_per_step() < 1e9          # fits the L2: flush it between steps
     main_flush = torch.zeros(96 * 1024 * 1024, dtype=torch.float32, device="cuda") if small else None
-    ms, launches, elements, alg_bytes, kernels = bench_workload(B, WL, wl, args.steps, args.warmup, dist, world, rank,
-                                                                sampler, flush=main_flush, profile=True)
+    ms, launches, elements, alg_bytes, kernels, per_step = bench_workload(B, WL, wl, args.steps, args.warmup, dist, world, rank,
+                                                                          sampler, flush=main_flush, profile=True)
     del main_flush
     clocks = sampler.finish()
-    peak, peak_kind = _measured_peak()
-    value = elements * args.steps / (ms * 1e-3)
     step_gbs = alg_bytes * args.steps / (ms * 1e-3) / 1e9
-    top = max(kernels, key=lambda kk: kk["ms_per_launch"] * kk["launches"])      # the dominant kernel
-    achieved = top["GB/s"] if top["GB/s"] is not None else step_gbs
-    traffic = None
-    if (NCU_TRAFFIC_BYTES_PER_ELEMENT is not None and NCU_TRAFFIC_KERNEL_SHA256 == _kernel_hash()
-            and top["algorithmic_bytes_per_launch"]):
-        traffic = NCU_TRAFFIC_BYTES_PER_ELEMENT * top["algorithmic_bytes_per_launch"] / 20.0
-    line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": workload_config(wl, world),
-        "gpu_launches": launches, "clocks": clocks,
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": traffic, "peak_kind": "of %s" % peak_kind, "frac_of_8000_nominal": achieved / 8000.0,
-                     "kernel": top["kernel"], "algorithmic_bytes_per_launch": top["algorithmic_bytes_per_launch"],
-                     "launch_ms": top["ms_per_launch"],
-                     "whole_step": {"GB/s": step_gbs, "frac": step_gbs / peak, "frac_of_8000_nominal": step_gbs / 8000.0,
-                                    "algorithmic_bytes_per_step": alg_bytes, "launches_per_step": launches / args.steps},
-                     "kernels": kernels,
-                     "note": "per-kernel times from a second pass of the same steps with each launch bracketed by "
-                             "CUDA events on the launching stream; whole_step is the timed region itself"},
-    }
+    line.update({"value": elements * args.steps / (ms * 1e-3), "ms_per_step": ms / args.steps, **step_spread(per_step),
+                 "gpu_launches": launches, "clocks": clocks,
+                 "roofline": roofline_of(kernels, step_gbs, alg_bytes, launches / args.steps, peak, peak_kind)})
 
     if args.no_extras and args.aux and world == 1:
         line["aux"] = bench_aux(B, WL, wl)
@@ -586,16 +705,18 @@ def main():
                      if not (r == wl.ratio and v == wl.variant)]
             for w in todo:
                 small = w.algorithmic_bytes_per_step() < 1e9
-                ms_w, launches_w, el_w, bytes_w, _ = bench_workload(B, WL, w, w.steps, 3, None, 1, 0,
-                                                                    flush=flush if small else None)
+                ms_w, launches_w, el_w, bytes_w, _, per_w = bench_workload(B, WL, w, w.steps, 3, None, 1, 0,
+                                                                           flush=flush if small else None)
                 gbs = bytes_w * w.steps / (ms_w * 1e-3) / 1e9
                 resident = None
                 if small:      # the whole state fits the L2: also the back-to-back time without a flush ("effective")
-                    ms_r, _, _, _, _ = bench_workload(B, WL, w, w.steps, 3, None, 1, 0, flush=None)
-                    resident = {"ms_per_step": ms_r / w.steps, "effective_GB/s": bytes_w * w.steps / (ms_r * 1e-3) / 1e9,
+                    ms_r, _, _, _, _, per_r = bench_workload(B, WL, w, w.steps, 3, None, 1, 0, flush=None)
+                    resident = {"ms_per_step": ms_r / w.steps, **step_spread(per_r),
+                                "effective_GB/s": bytes_w * w.steps / (ms_r * 1e-3) / 1e9,
                                 "note": "state stays in the 126 MB L2 between steps: not an HBM figure"}
                 per.append({"cfg": w.cfg, "name": w.name, "ratio": w.ratio, "variant": WL.VARIANT_NAMES[w.variant],
-                            "steps": w.steps, "ms_per_step": ms_w / w.steps, "elements_per_s": el_w * w.steps / (ms_w * 1e-3),
+                            "steps": w.steps, "ms_per_step": ms_w / w.steps, **step_spread(per_w),
+                            "elements_per_s": el_w * w.steps / (ms_w * 1e-3),
                             "GB/s": gbs, "frac_of_measured_peak": gbs / peak, "frac_of_8000_nominal": gbs / 8000.0,
                             "launches_per_step": launches_w / w.steps, "l2_resident": resident,
                             "l2": "flushed between steps" if small else "inputs larger than L2"})
@@ -604,9 +725,7 @@ def main():
             line["per_config"] = per
             line["per_config_note"] = ("EF, DEF and DEF-A run the same kernels given the gradients: the variant changes only "
                                        "where the caller evaluates them and the returned model")
-            v, sec, n = oracle_sample_run(WL, wl, 3, 1, budget_s=20.0)
-            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle",
-                                    "sample": "3 oracle steps on columns [0, %d) of d = %d, W = %d (%.1f s)" % (n, wl.d, wl.W, sec)}
+            line["cpu_baseline"] = cpu_baseline(wl, 20, 1)
     if rank == 0:
         print(json.dumps(line))
     if dist is not None:

@@ -376,8 +376,9 @@ def_step_stream_kernel(const StepArgs a) {
 // k / TILE + 4 CTAs covers every case.  CTA i takes the i-th touched tile: first those of
 // the run that starts at s, then those of the wrapped run [0, s + k - d) that the first
 // run has not already covered.  CTAs beyond the last touched tile leave.
-template <bool MOM, int U, int POL, bool DETACH = false>
-__global__ void __launch_bounds__(kTileThreads)
+// MINB: CTAs per SM the compiler is asked to make room for (it caps the registers accordingly).
+template <bool MOM, int U, int POL, bool DETACH = false, int MINB = 3>
+__global__ void __launch_bounds__(kTileThreads, MINB)
 def_step_block_kernel(const StepArgs a) {
     // The stream kernel that follows in the stream works on other tiles and needs nothing from
     // this kernel: when it was launched with programmatic stream serialization, let its CTAs

@@ -32,12 +32,15 @@ def test_touched_columns_against_brute_force():
 
 def test_reference_arm_prints_the_contract_line():
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "2",
-                          "--warmup", "3", "--reference-budget-s", "3"], capture_output=True, text=True, timeout=300)
+                          "--warmup", "3", "--reference-columns", "200000"], capture_output=True, text=True, timeout=300)
     assert out.returncode == 0, out.stderr
     line = json.loads(out.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["unit"] == "elements/s" and line["higher_is_better"] is True
     assert line["value"] > 0 and line["steps"] == 2 and line["vs_baseline"] is None
-    assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] == 1
+    base = line["cpu_baseline"]
+    assert base["kind"] == "oracle" and base["cores"] >= 1 and base["value"] == line["value"]
+    assert base["one_core"]["cores"] == 1 and base["one_core"]["value"] > 0     # the plain build, same sample
+    assert "[0, 200000)" in base["sample"]
     assert line["e2e"]["value"] == line["value"] and line["e2e"]["h2d_bytes_per_step"] == 0
     assert "cfg5" in line["config"]["workload"]
     # other ranks of a multi-process launch do no work and print nothing

@@ -300,6 +300,16 @@ int def_set_compressor(def_ctx *ctx, int32_t compressor, float delta);
  */
 int def_set_small_step_bytes(def_ctx *ctx, int64_t bytes);
 
+/*
+ * Whether the second kernel of a pair may start while the first (the tiles that touch the block)
+ * is still running -- they write disjoint floats, and work enqueued after the pair is ordered
+ * behind both either way.  DEF_OVERLAP_AUTO (default) lets the library decide from the sizes,
+ * DEF_OVERLAP_NEVER runs the two one after the other, DEF_OVERLAP_ALWAYS side by side.
+ * Results are bit-identical in every mode.
+ */
+enum { DEF_OVERLAP_AUTO = 0, DEF_OVERLAP_NEVER = 1, DEF_OVERLAP_ALWAYS = 2 };
+int def_set_pair_overlap(def_ctx *ctx, int32_t mode);
+
 /* Learning-rate schedules: eta may change between steps. */
 int def_set_lr(def_ctx *ctx, float lr);
 
@@ -330,6 +340,16 @@ int def_block_start_device(const uint64_t *seeds, const uint64_t *steps, const i
 enum { DEF_KERNEL_STREAM = 0, DEF_KERNEL_BLOCK = 1, DEF_KERNEL_GENERAL = 2, DEF_KERNEL_KINDS = 3 };
 int def_set_kernel_timing(def_ctx *ctx, int enable);
 int def_kernel_time(const def_ctx *ctx, int kernel, double *total_ms_out, int64_t *launches_out);
+
+/*
+ * How a step with (step, seed) on local coordinates [j0, j0 + n) is cut between the two kernels of
+ * a pair, computed on the host from the same block start the kernels draw.  Tiles are runs of 1024
+ * local coordinates.  The tiles that touch the block (Section 1's k coordinates from s, wrapping
+ * mod d) are tiles [0, plan_out[2]) and [plan_out[0], plan_out[0] + plan_out[1]), disjoint; the
+ * block kernel gets one CTA for each, the stream kernel CTAs for the other plan_out[3] tiles.
+ * n >= 1.  Touches no GPU.
+ */
+int def_tile_plan(const def_ctx *ctx, int64_t j0, int64_t n, uint64_t step, uint64_t seed, int64_t plan_out[4]);
 
 /* Kernels this context has launched so far (every launch of every call). */
 int def_launch_count(const def_ctx *ctx, int64_t *count_out);

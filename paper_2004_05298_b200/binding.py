@@ -43,9 +43,11 @@ SIGNATURES = {
     "def_set_lr": (ctypes.c_int, [_ptr, _f32]),
     "def_set_small_step_bytes": (ctypes.c_int, [_ptr, _i64]),
     "def_set_compressor": (ctypes.c_int, [_ptr, _i32, _f32]),
+    "def_set_pair_overlap": (ctypes.c_int, [_ptr, _i32]),
     "def_block_start": (ctypes.c_int, [_ptr, _u64, _u64, _ptr]),
     "def_block_start_device": (ctypes.c_int, [_ptr, _ptr, _ptr, _i64, _ptr, _ptr]),
     "def_launch_count": (ctypes.c_int, [_ptr, _ptr]),
+    "def_tile_plan": (ctypes.c_int, [_ptr, _i64, _i64, _u64, _u64, _ptr]),
     "def_set_kernel_timing": (ctypes.c_int, [_ptr, ctypes.c_int]),
     "def_kernel_time": (ctypes.c_int, [_ptr, ctypes.c_int, _ptr, _ptr]),
     "def_last_error": (ctypes.c_char_p, []),
@@ -197,6 +199,13 @@ def def_block_start_device(seeds, steps, ds, starts_out, stream=None):
                                       ctypes.c_void_p(raw)))
 
 
+def def_tile_plan(ctx, j0, n, step, seed):
+    """(first tile of run A, its tiles, tiles of run B from tile 0, tiles left to the stream kernel)."""
+    out = (ctypes.c_int64 * 4)()
+    _check(lib.def_tile_plan(ctx.handle, int(j0), int(n), int(step), int(seed), out))
+    return tuple(int(v) for v in out)
+
+
 def def_launch_count(ctx):
     out = ctypes.c_int64(0)
     _check(lib.def_launch_count(ctx.handle, ctypes.byref(out)))
@@ -271,6 +280,13 @@ def def_step_columns_detach(ctx, j0, n, ld, params, grads, errors, mom, detached
 
 def def_set_small_step_bytes(ctx, nbytes):
     _check(lib.def_set_small_step_bytes(ctx.handle, int(nbytes)))
+
+
+DEF_OVERLAP_AUTO, DEF_OVERLAP_NEVER, DEF_OVERLAP_ALWAYS = 0, 1, 2
+
+
+def def_set_pair_overlap(ctx, mode):
+    _check(lib.def_set_pair_overlap(ctx.handle, int(mode)))
 
 
 def def_set_compressor(ctx, compressor, delta=0.0):

@@ -46,6 +46,7 @@ struct def_ctx {
     cudaStream_t stream = nullptr;
     int64_t launches = 0;
     int64_t small_step_bytes = 0;  // set by def_create (kSmallStepBytesDefault)
+    int32_t pair_overlap = DEF_OVERLAP_AUTO;
     int32_t compressor = DEF_COMPRESSOR_RBGS;
     float delta = 0.f;             // factor of DEF_COMPRESSOR_SCALE
     // per-kernel device times (profiling aid, off by default)
@@ -186,6 +187,12 @@ cudaError_t counted_launch(def_ctx *ctx, int kind, cudaStream_t stream, Launch l
 // behind the stream kernel, is ordered behind both.  Not used in timing mode, where each
 // kernel is measured alone, nor when the block kernel went to another stream (`beside` false:
 // the two then overlap as work on two streams does).
+bool overlap_allowed(const def_ctx *ctx, const defk::StepArgs &a) {
+    (void)a;
+    if (ctx->pair_overlap == DEF_OVERLAP_NEVER) return false;
+    return true;
+}
+
 template <typename Kernel>
 cudaError_t launch_beside_block_kernel(const def_ctx *ctx, Kernel kernel, dim3 grid, unsigned threads,
                                        cudaStream_t stream, const defk::StepArgs &a, bool beside = true) {
@@ -195,7 +202,7 @@ cudaError_t launch_beside_block_kernel(const def_ctx *ctx, Kernel kernel, dim3 g
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = (ctx->timing || !beside) ? 0 : 1;
+    attr[0].val.programmaticStreamSerializationAllowed = (ctx->timing || !beside || !overlap_allowed(ctx, a)) ? 0 : 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, a);
@@ -236,16 +243,21 @@ cudaError_t launch_one(def_ctx *ctx, const defk::StepArgs &a, cudaStream_t strea
     if (V == 4 && 20 * (int64_t)a.W * a.n >= ctx->small_step_bytes) {
         const int64_t tiles = (a.n + defk::kTile - 1) / defk::kTile;
         if (tiles > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+        // Each kernel gets CTAs for its own tiles only.  The host draws the block start with the
+        // same function the kernels use (they still draw it themselves) to count them.
+        const defk::TouchedTiles touched = defk::touched_tiles(a, defk::block_start(a.seed, a.step, a.d));
+        const int64_t block_ctas = touched.a_count + touched.b_count;
+        const int64_t stream_tiles = tiles - block_ctas;
         // the few tiles that touch the block first, then the stream over all the others
-        const int64_t block_ctas = a.k / defk::kTile + 4;
-        const unsigned block_grid = (unsigned)(block_ctas < tiles + 1 ? block_ctas : tiles + 1);
+        const unsigned block_grid = (unsigned)(block_ctas > 0 ? block_ctas : 1);
         const bool beside = block_stream == stream;
         cudaError_t err = counted_launch(ctx, DEF_KERNEL_BLOCK, block_stream, [&] {
             defk::def_step_block_kernel<MOM, kBlockRows, kPolicy, DETACH><<<block_grid, defk::kTileThreads, 0, block_stream>>>(a);
         });
         if (err != cudaSuccess) return err;
         constexpr int kStreamTiles = 2;
-        const int64_t slots = (tiles + kStreamTiles - 1) / kStreamTiles;
+        int64_t slots = (stream_tiles + kStreamTiles - 1) / kStreamTiles;
+        if (slots < 1) slots = 1;                       // k = d: nothing to stream; one idle CTA keeps the pair a pair
         if constexpr (DETACH) {
             const int64_t segments = (slots + kDetachChunkCtas - 1) / kDetachChunkCtas;
             const int64_t ctas = segments * kDetachChunkCtas * a.W;
@@ -489,6 +501,19 @@ int def_block_start_device(const uint64_t *seeds, const uint64_t *steps, const i
     return DEF_OK;
 }
 
+int def_tile_plan(const def_ctx *ctx, int64_t j0, int64_t n, uint64_t step, uint64_t seed, int64_t plan_out[4]) {
+    if (!ctx || !plan_out) return fail(DEF_ERR_NULL, "ctx and plan_out must not be NULL");
+    if (j0 < 0 || n < 1 || j0 > ctx->d || n > ctx->d - j0)
+        return fail(DEF_ERR_ARG, "column range [%lld, %lld) is outside [0, %lld) or empty", (long long)j0,
+                    (long long)(j0 + n), (long long)ctx->d);
+    defk::StepArgs a = {};
+    a.n = n; a.d = ctx->d; a.j0 = j0; a.k = ctx->k;
+    const defk::TouchedTiles t = defk::touched_tiles(a, defk::block_start(seed, step, ctx->d));
+    plan_out[0] = t.a_first; plan_out[1] = t.a_count; plan_out[2] = t.b_count;
+    plan_out[3] = (n + defk::kTile - 1) / defk::kTile - t.a_count - t.b_count;
+    return DEF_OK;
+}
+
 int def_launch_count(const def_ctx *ctx, int64_t *count_out) {
     if (!ctx || !count_out) return fail(DEF_ERR_NULL, "ctx and count_out must not be NULL");
     *count_out = ctx->launches;
@@ -512,6 +537,14 @@ int def_set_small_step_bytes(def_ctx *ctx, int64_t bytes) {
     if (!ctx) return fail(DEF_ERR_NULL, "ctx is NULL");
     if (bytes < 0) return fail(DEF_ERR_ARG, "bytes must be >= 0");
     ctx->small_step_bytes = bytes;
+    return DEF_OK;
+}
+
+int def_set_pair_overlap(def_ctx *ctx, int32_t mode) {
+    if (!ctx) return fail(DEF_ERR_NULL, "ctx is NULL");
+    if (mode != DEF_OVERLAP_AUTO && mode != DEF_OVERLAP_NEVER && mode != DEF_OVERLAP_ALWAYS)
+        return fail(DEF_ERR_ARG, "unknown overlap mode %d", mode);
+    ctx->pair_overlap = mode;
     return DEF_OK;
 }
 

@@ -302,29 +302,61 @@ def_step_kernel(const StepArgs a) {
 constexpr int kTileThreads = 256;
 constexpr int64_t kTile = (int64_t)kTileThreads * 4;
 
-__device__ __forceinline__ bool tile_touches_block(const StepArgs &a, int64_t s, int64_t tile) {
-    const int64_t tile0 = tile * kTile;
-    const int64_t tile_len = (a.n - tile0 < kTile) ? a.n - tile0 : kTile;
-    int64_t off0 = a.j0 + tile0 - s;                 // offset of the tile's start from s, mod d
-    if (off0 < 0) off0 += a.d;
-    return off0 < a.k || off0 + tile_len > a.d;      // starts inside the block, or wraps onto its start
+// The tiles of the local range [j0, j0 + n) that touch the block {(s + i) mod d : i < k}.  The
+// block is at most two runs of local coordinates (it may wrap past d, and the local range may cut
+// it): run A = [s, min(s + k, d)) and, if the block wraps, run B = [0, s + k - d), both clipped to
+// the local range.  B ends before s, so its tiles lie at or before A's first tile; a tile both
+// runs reach counts for A.  Touched tiles are therefore tiles [0, b_count) and
+// [a_first, a_first + a_count), disjoint and in this order.  (Host and device: the host sizes the
+// grids from the same arithmetic.)
+struct TouchedTiles {
+    int64_t a_first, a_count, b_count;
+};
+
+__host__ __device__ __forceinline__ TouchedTiles touched_tiles(const StepArgs &a, int64_t s) {
+    const int64_t lo = a.j0, hi = a.j0 + a.n;
+    const int64_t a0 = s > lo ? s : lo;
+    int64_t a1 = s + a.k < a.d ? s + a.k : a.d;
+    a1 = a1 < hi ? a1 : hi;
+    int64_t b1 = s + a.k - a.d;                                  // <= s; > 0 only if the block wraps
+    b1 = b1 < hi ? b1 : hi;
+    TouchedTiles t;
+    t.a_first = 0; t.a_count = 0; t.b_count = 0;
+    if (a1 > a0) {
+        t.a_first = (a0 - lo) / kTile;
+        t.a_count = (a1 - 1 - lo) / kTile - t.a_first + 1;
+    }
+    if (b1 > lo) {
+        t.b_count = (b1 - 1 - lo) / kTile + 1;
+        if (t.a_count > 0 && t.b_count > t.a_first) t.b_count = t.a_first;
+    }
+    return t;
+}
+
+// The u-th tile (in increasing order) that does NOT touch the block: skip the two runs.
+__host__ __device__ __forceinline__ int64_t untouched_tile(const TouchedTiles &t, int64_t u) {
+    int64_t tile = u + t.b_count;
+    if (t.a_count > 0 && tile >= t.a_first) tile += t.a_count;
+    return tile;
 }
 
 // Tiles that do not touch the block (all but about k / TILE + 2 of them) have nothing to
-// sum: C(p) = 0 and e' = p.  The grid is (tiles, W) and CTA (t, w) does worker w's row of
-// tile t: three 16-byte loads and two stores per thread, few registers, full occupancy.
-// Consecutive CTAs sweep one row after the other, so the memory system sees a handful of
-// long sequential streams.  CTAs of tiles that touch the block store nothing.
+// sum: C(p) = 0 and e' = p.  CTA (i, w) does worker w's row of the i-th such tiles: three 16-byte
+// loads and two stores per thread, few registers, full occupancy.  The grid holds CTAs for these
+// tiles only -- the host sizes it from the same block start -- so no CTA is launched just to
+// find that its tile belongs to the other kernel (with k = d/8 those were an eighth of the
+// grid and cost 2 % of the step).  Consecutive CTAs sweep one row after the other, so the memory
+// system sees a handful of long sequential streams.
 // With DETACH the kernel also writes z_w = x - lambda e'_w for its row (x is unchanged outside
 // the block), which makes x a sixth stream that every worker's CTA of a tile reads.  ORDER
 // chooses how CTAs are numbered, i.e. what runs together:
-//   kOrderRows     grid (tiles, W): row after row, the flat stream.  (With DETACH, x would be
+//   kOrderRows     grid (tile slots, W): row after row, the flat stream.  (With DETACH, x would be
 //                  re-read from HBM for every row: it is far larger than the L2.)
 //   kOrderChunked  1-D grid: a.chunk consecutive CTAs sweep a segment of row 0, the next a.chunk
 //                  the same segment of row 1, ...; then the next segment.  Long sequential
 //                  streams, and the segment of x stays in the L2 until the last row has used it.
 // TILES CTAs' worth of tiles share one CTA of TILES * kTileThreads threads (each group of
-// kTileThreads threads still owns one tile and decides for it alone).
+// kTileThreads threads still owns one tile).
 constexpr int kOrderRows = 0, kOrderChunked = 1;
 
 template <bool MOM, int POL, bool DETACH = false, int ORDER = kOrderRows, int TILES = 1>
@@ -341,14 +373,14 @@ def_step_stream_kernel(const StepArgs a) {
         w = (unsigned)(rem / a.chunk);
         first = segment * a.chunk + rem % a.chunk;
     }
-    const int64_t tile = first * TILES + (int64_t)(threadIdx.x / kTileThreads);
-    const int64_t col = tile * kTile + (int64_t)(threadIdx.x % kTileThreads) * 4;
-    const bool live = col < a.n;
-    const size_t at = (size_t)w * (size_t)a.ld + (size_t)col;
-    // (Issuing the loads before the CTA learns the block start -- they do not depend on it -- was
-    // measured 2 % slower on the largest workload and no faster on the small ones.)
+    // (Issuing the loads before the CTA learns the block start is not possible here -- which tile
+    // a thread owns depends on it -- and was slower when it was: see the design-variants program.)
     const int64_t s = cta_block_start(a);
-    if (live && !tile_touches_block(a, s, tile)) {
+    const TouchedTiles touched = touched_tiles(a, s);
+    const int64_t tile = untouched_tile(touched, first * TILES + (int64_t)(threadIdx.x / kTileThreads));
+    const int64_t col = tile * kTile + (int64_t)(threadIdx.x % kTileThreads) * 4;
+    if (col < a.n) {                                   // (slots past the last untouched tile land beyond n)
+        const size_t at = (size_t)w * (size_t)a.ld + (size_t)col;
         const Vec<4> g = load_vec<4, POL>(a.g + at);
         const Vec<4> e = load_vec<4, POL>(a.e + at);
         Vec<4> m, x;
@@ -371,11 +403,9 @@ def_step_stream_kernel(const StepArgs a) {
 }
 
 // Tiles that touch the block: one CTA per tile walks the W rows in order (column_group).
-// The block is at most two runs of local coordinates (it may wrap past d, and the local
-// range may cut it); a run of length L touches at most L / TILE + 2 tiles, so a grid of
-// k / TILE + 4 CTAs covers every case.  CTA i takes the i-th touched tile: first those of
-// the run that starts at s, then those of the wrapped run [0, s + k - d) that the first
-// run has not already covered.  CTAs beyond the last touched tile leave.
+// A run of length L touches at most L / TILE + 2 tiles, so a grid of k / TILE + 4 CTAs covers
+// every case.  CTA i takes the i-th touched tile: first those of run A, then those of run B.
+// CTAs beyond the last touched tile leave.
 // MINB: CTAs per SM the compiler is asked to make room for (it caps the registers accordingly).
 template <bool MOM, int U, int POL, bool DETACH = false, int MINB = 3>
 __global__ void __launch_bounds__(kTileThreads, MINB)
@@ -385,23 +415,13 @@ def_step_block_kernel(const StepArgs a) {
     // start now instead of after this grid has drained (a no-op otherwise).
     release_dependent_grids();
     const int64_t s = cta_block_start(a);
-    // the two runs in model coordinates, clipped to the local range [j0, j0 + n)
-    const int64_t lo = a.j0, hi = a.j0 + a.n;
-    int64_t a0 = s > lo ? s : lo;                                // run A = [s, min(s + k, d))
-    int64_t a1 = (s + a.k < a.d ? s + a.k : a.d);
-    a1 = a1 < hi ? a1 : hi;
-    int64_t b0 = lo;                                             // run B = [0, s + k - d)
-    int64_t b1 = s + a.k - a.d;
-    b1 = b1 < hi ? b1 : hi;
-    const int64_t tA0 = (a0 - lo) / kTile, tA1 = a1 > a0 ? (a1 - 1 - lo) / kTile : tA0 - 1;
-    const int64_t tB0 = 0, tB1 = b1 > b0 ? (b1 - 1 - lo) / kTile : -1;
-    const int64_t nA = tA1 - tA0 + 1;
+    const TouchedTiles touched = touched_tiles(a, s);
     int64_t tile;
-    if ((int64_t)blockIdx.x < nA) {
-        tile = tA0 + blockIdx.x;
+    if ((int64_t)blockIdx.x < touched.a_count) {
+        tile = touched.a_first + blockIdx.x;
     } else {
-        tile = tB0 + ((int64_t)blockIdx.x - nA);
-        if (tile > tB1 || (tile >= tA0 && tile <= tA1)) return;  // past the end, or already done as part of run A
+        tile = (int64_t)blockIdx.x - touched.a_count;
+        if (tile >= touched.b_count) return;
     }
     const int64_t col = tile * kTile + (int64_t)threadIdx.x * 4;
     if (col < a.n) column_group<4, MOM, U, POL, DETACH>(a, s, col);

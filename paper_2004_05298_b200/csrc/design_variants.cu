@@ -8,9 +8,10 @@
 //     the same with evict-first cache hints, 256-bit accesses, a persistent grid-stride loop,
 //     one thread walking all W rows of its columns, and 1-D bulk asynchronous copies through
 //     shared memory;
-//   * the library's own stream kernel as shipped, and two changes to how it learns the block
-//     start (loads issued before the CTA-wide hand-over; the start passed in by the host, which
-//     is the bound on what hiding that latency can gain);
+//   * the library's own stream kernel as shipped, and a stream kernel whose grid covers all tiles
+//     (CTAs of tiles that touch the block idle) with the block start obtained in three ways:
+//     per CTA before the loads, per CTA after the loads have been issued, and passed in by the
+//     host, which is the bound on what hiding that latency can gain;
 //   * the library's block kernel (tiles that touch the block) for 2 / 4 / 8 rows in flight and
 //     1..4 CTAs per SM requested from the compiler.
 // Every kernel here does the arithmetic of the step; none is timed with work left out.
@@ -173,9 +174,20 @@ bulk_kernel(const float *__restrict__ g, float *__restrict__ e, float *__restric
     }
 }
 
-// ---- the library's stream kernel with the block start obtained in other ways ------------------
-// MODE 1: the three loads are issued before the CTA-wide hand-over of the block start.
+// ---- a stream kernel over ALL tiles, with the block start obtained in three ways ---------------
+// Grid (tile pairs, W) over every tile; a CTA whose tile touches the block stores nothing (the
+// library's kernel before its grid was cut down to the tiles it works on).
+// MODE 0: block start per CTA (Philox by one thread, handed over through shared memory), then loads.
+// MODE 1: the three loads are issued before that hand-over.
 // MODE 2: the start is a kernel argument (no Philox, no barrier) -- what hiding the latency can gain at most.
+__device__ __forceinline__ bool tile_touches_block(const StepArgs &a, int64_t s, int64_t tile) {
+    const int64_t tile0 = tile * defk::kTile;
+    const int64_t tile_len = (a.n - tile0 < defk::kTile) ? a.n - tile0 : defk::kTile;
+    int64_t off0 = a.j0 + tile0 - s;                 // offset of the tile's start from s, mod d
+    if (off0 < 0) off0 += a.d;
+    return off0 < a.k || off0 + tile_len > a.d;      // starts inside the block, or wraps onto its start
+}
+
 template <int MODE>
 __global__ void __launch_bounds__(512)
 stream_variant_kernel(const StepArgs a, int64_t s_from_host) {
@@ -188,7 +200,7 @@ stream_variant_kernel(const StepArgs a, int64_t s_from_host) {
         g = defk::load_vec<4, 0>(a.g + at); e = defk::load_vec<4, 0>(a.e + at); m = defk::load_vec<4, 0>(a.m + at);
     }
     const int64_t s = MODE == 2 ? s_from_host : defk::cta_block_start(a);
-    if (live && !defk::tile_touches_block(a, s, tile)) {
+    if (live && !tile_touches_block(a, s, tile)) {
         if (MODE != 1) {
             g = defk::load_vec<4, 0>(a.g + at); e = defk::load_vec<4, 0>(a.e + at); m = defk::load_vec<4, 0>(a.m + at);
         }
@@ -292,7 +304,9 @@ int main(int argc, char **argv) {
     }
     const double bytes_stream = 20.0 * (double)W * (double)(d - touched);
     const double bytes_block = 20.0 * (double)W * (double)touched + 8.0 * (double)k;
-    const unsigned block_grid = (unsigned)(k / defk::kTile + 4 < tiles + 1 ? k / defk::kTile + 4 : tiles + 1);
+    const defk::TouchedTiles tt = defk::touched_tiles(a, s0);
+    const unsigned block_grid = (unsigned)(tt.a_count + tt.b_count > 0 ? tt.a_count + tt.b_count : 1);
+    const dim3 stream_grid((unsigned)((tiles - tt.a_count - tt.b_count + 1) / 2 > 0 ? (tiles - tt.a_count - tt.b_count + 1) / 2 : 1), (unsigned)W);
 
     Timer timer;
     if (cold) {                                        // 384 MB, three times the L2
@@ -328,11 +342,13 @@ int main(int argc, char **argv) {
     }
     row("1-D bulk async copies through shared memory (16 KB chunks)", bytes_all,
         [&] { bulk_kernel<<<(unsigned)((n + kBulkFloats - 1) / kBulkFloats), kBulkThreads, 3 * kBulkFloats * 4>>>(g, e, m, n, eta, mu, gave_up); });
-    row("library stream kernel as shipped (block start per CTA, then loads)", bytes_stream,
-        [&] { defk::def_step_stream_kernel<true, 0, false, defk::kOrderRows, 2><<<pair_grid, 512>>>(a); });
-    row("stream kernel, loads issued before the block start is known", bytes_stream,
+    row("library stream kernel as shipped (grid over the tiles outside the block only)", bytes_stream,
+        [&] { defk::def_step_stream_kernel<true, 0, false, defk::kOrderRows, 2><<<stream_grid, 512>>>(a); });
+    row("stream kernel over all tiles, block start per CTA, then loads", bytes_stream,
+        [&] { stream_variant_kernel<0><<<pair_grid, 512>>>(a, s0); });
+    row("stream kernel over all tiles, loads issued before the block start is known", bytes_stream,
         [&] { stream_variant_kernel<1><<<pair_grid, 512>>>(a, s0); });
-    row("stream kernel, block start passed in by the host (bound)", bytes_stream,
+    row("stream kernel over all tiles, block start passed in by the host (bound)", bytes_stream,
         [&] { stream_variant_kernel<2><<<pair_grid, 512>>>(a, s0); });
     row("library block kernel, U = 2 rows in flight, min 1 CTA/SM", bytes_block, [&] { launch_block<2, 1>(a, block_grid); });
     row("library block kernel, U = 2, min 4 CTAs/SM", bytes_block, [&] { launch_block<2, 4>(a, block_grid); });

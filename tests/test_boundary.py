@@ -124,3 +124,38 @@ def test_host_block_start_matches_oracle():
                 seed, step = seed % 6, step % 128
             assert B.def_block_start(ctx, step, seed) == oracle.block_start(seed, step, d)
         B.def_destroy(ctx)
+
+
+def test_tile_plan_against_brute_force():
+    """The cut of a step's tiles between the two kernels of a pair (host arithmetic the grids are
+    sized from): against the set of tiles that hold a block coordinate, found by enumeration, with
+    the block start taken from the oracle's sampler."""
+    import random
+    rnd = random.Random(5)
+    TILE = 1024
+    cases = 0
+    for _ in range(400):
+        d = rnd.choice([rnd.randint(1, 50), rnd.randint(50, 5000), rnd.randint(5000, 40000)])
+        k = rnd.choice([1, d, max(1, d - 1), rnd.randint(1, d)])
+        ctx = B.def_create(d, 2, k, 0, 0.1, 0.9)
+        for step in range(6):
+            seed = rnd.randrange(100)
+            j0 = rnd.choice([0, rnd.randrange(d)])
+            n = rnd.choice([d - j0, rnd.randint(1, d - j0)])
+            s = oracle.block_start(seed, step, d)
+            block = {(s + i) % d for i in range(k)}
+            want = sorted({(j - j0) // TILE for j in block if j0 <= j < j0 + n})
+            a_first, a_count, b_count, rest = B.def_tile_plan(ctx, j0, n, step, seed)
+            got = list(range(b_count)) + list(range(a_first, a_first + a_count))
+            assert a_count == 0 or b_count <= a_first, (d, k, s, j0, n)
+            assert got == want, (d, k, s, j0, n, got[:5], want[:5])
+            assert rest == -(-n // TILE) - len(want)
+            cases += 1
+        B.def_destroy(ctx)
+    assert cases == 2400
+    ctx = B.def_create(100, 2, 10, 0, 0.1, 0.9)
+    out = (ctypes.c_int64 * 4)()
+    assert B.lib.def_tile_plan(ctx.handle, 0, 0, 0, 0, out) == B.DEF_ERR_ARG
+    assert B.lib.def_tile_plan(ctx.handle, 50, 51, 0, 0, out) == B.DEF_ERR_ARG
+    assert B.lib.def_tile_plan(ctx.handle, 0, 100, 0, 0, None) == B.DEF_ERR_NULL
+    B.def_destroy(ctx)

@@ -209,11 +209,11 @@ cudaError_t launch_beside_block_kernel(const def_ctx *ctx, Kernel kernel, dim3 g
 }
 
 // With the fused detach output x becomes a stream every worker's CTA of a tile reads.  The
-// stream kernel then runs in chunked order: 256 CTAs (two tiles each: 2 MB of every row and
-// of x) sweep a segment of row 0, the next 256 the same segment of row 1, and so on, so the
-// streams stay long and sequential while the segment of x stays in the L2 for all W rows.
-// Measured on the VGG-16-sized workload: 8.12 ms, against 8.78 ms with the W CTAs of a tile
-// adjacent and 8.97 ms row after row (x re-read from HBM for every row).
+// stream kernel then runs in chunked order: 256 CTAs (four tiles each with momentum: 4 MB of
+// every row and of x) sweep a segment of row 0, the next 256 the same segment of row 1, and so
+// on, so the streams stay long and sequential while the segment of x stays in the L2 for all W
+// rows.  Measured on the VGG-16-sized workload: 7.91 ms, against 8.78 ms with the W CTAs of a
+// tile adjacent and 8.97 ms row after row (x re-read from HBM for every row).
 constexpr int kDetachChunkCtas = 256;
 
 // Steps that move fewer bytes than this run as ONE launch of the general kernel instead of the
@@ -255,7 +255,12 @@ cudaError_t launch_one(def_ctx *ctx, const defk::StepArgs &a, cudaStream_t strea
             defk::def_step_block_kernel<MOM, kBlockRows, kPolicy, DETACH><<<block_grid, defk::kTileThreads, 0, block_stream>>>(a);
         });
         if (err != cudaSuccess) return err;
-        constexpr int kStreamTiles = 2;
+        // Tiles per CTA of the stream kernel, i.e. CTAs of 256 times this many threads, two or four
+        // of them resident per SM.  With momentum (3 loads, 2 stores per thread) CTAs of 1024
+        // threads ran the VGG-16-, ResNet-50- and ResNet-18-sized steps 1.2 / 0.9 / 0.7 % faster than
+        // CTAs of 512, and the step with the detach output 0.9 %; without momentum (2 loads, 1 store)
+        // they ran it 5 % slower, and CTAs of 768 threads 15 % slower.
+        constexpr int kStreamTiles = MOM ? 4 : 2;
         int64_t slots = (stream_tiles + kStreamTiles - 1) / kStreamTiles;
         if (slots < 1) slots = 1;                       // k = d: nothing to stream; one idle CTA keeps the pair a pair
         if constexpr (DETACH) {
@@ -270,8 +275,6 @@ cudaError_t launch_one(def_ctx *ctx, const defk::StepArgs &a, cudaStream_t strea
             });
         }
         else {
-            // two tiles per CTA of 512 threads: 0.4-0.9 % faster than one tile per 256 (half as
-            // many block-start computations), while 1024 threads lose 20 %
             const dim3 grid((unsigned)slots, (unsigned)a.W);
             return counted_launch(ctx, DEF_KERNEL_STREAM, stream, [&] {
                 launch_beside_block_kernel(ctx, defk::def_step_stream_kernel<MOM, kPolicy, false, defk::kOrderRows, kStreamTiles>,

@@ -373,10 +373,16 @@ def_step_stream_kernel(const StepArgs a) {
         w = (unsigned)(rem / a.chunk);
         first = segment * a.chunk + rem % a.chunk;
     }
-    // (Issuing the loads before the CTA learns the block start is not possible here -- which tile
-    // a thread owns depends on it -- and was slower when it was: see the design-variants program.)
-    const int64_t s = cta_block_start(a);
-    const TouchedTiles touched = touched_tiles(a, s);
+    // One thread draws the block start and works out which tiles touch the block; the others wait
+    // for the three numbers.  (Every thread doing that arithmetic itself after the hand-over of s
+    // cost the step without momentum, whose CTAs live shortest, 5 %, and the step with momentum
+    // 0.4 % at four tiles per CTA.  Issuing the loads before
+    // the hand-over is not possible here -- which tile a thread owns depends on it -- and was
+    // slower when it was: see the design-variants program.)
+    __shared__ TouchedTiles touched_shared;
+    if (threadIdx.x == 0) touched_shared = touched_tiles(a, block_start(a.seed, a.step, a.d));
+    __syncthreads();
+    const TouchedTiles touched = touched_shared;
     const int64_t tile = untouched_tile(touched, first * TILES + (int64_t)(threadIdx.x / kTileThreads));
     const int64_t col = tile * kTile + (int64_t)(threadIdx.x % kTileThreads) * 4;
     if (col < a.n) {                                   // (slots past the last untouched tile land beyond n)

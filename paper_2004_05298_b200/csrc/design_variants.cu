@@ -211,6 +211,21 @@ stream_variant_kernel(const StepArgs a, int64_t s_from_host) {
     }
 }
 
+// ---- the library's stream kernel with the tile plan handed in by the host: no per-CTA prologue ---
+template <int TILES>
+__global__ void __launch_bounds__(256 * TILES)
+stream_hostplan_kernel(const StepArgs a, const defk::TouchedTiles touched) {
+    const int64_t tile = defk::untouched_tile(touched, (int64_t)blockIdx.x * TILES + (int64_t)(threadIdx.x / defk::kTileThreads));
+    const int64_t col = tile * defk::kTile + (int64_t)(threadIdx.x % defk::kTileThreads) * 4;
+    if (col >= a.n) return;
+    const size_t at = (size_t)blockIdx.y * (size_t)a.ld + (size_t)col;
+    const Vec<4> g = defk::load_vec<4, 0>(a.g + at), e = defk::load_vec<4, 0>(a.e + at), m = defk::load_vec<4, 0>(a.m + at);
+    Vec<4> mn, en;
+    stream_math(g.v, e.v, m.v, a.eta, a.mu, mn.v, en.v);
+    defk::store_vec<4, 0>(a.m + at, mn);
+    defk::store_vec<4, 0>(a.e + at, en);
+}
+
 __global__ void empty_kernel() {}
 
 // Device time per launch.  Back to back (one event pair around `reps` launches), or -- with a
@@ -306,7 +321,7 @@ int main(int argc, char **argv) {
     const double bytes_block = 20.0 * (double)W * (double)touched + 8.0 * (double)k;
     const defk::TouchedTiles tt = defk::touched_tiles(a, s0);
     const unsigned block_grid = (unsigned)(tt.a_count + tt.b_count > 0 ? tt.a_count + tt.b_count : 1);
-    const dim3 stream_grid((unsigned)((tiles - tt.a_count - tt.b_count + 1) / 2 > 0 ? (tiles - tt.a_count - tt.b_count + 1) / 2 : 1), (unsigned)W);
+    const dim3 stream_grid((unsigned)((tiles - tt.a_count - tt.b_count + 3) / 4 > 0 ? (tiles - tt.a_count - tt.b_count + 3) / 4 : 1), (unsigned)W);
 
     Timer timer;
     if (cold) {                                        // 384 MB, three times the L2
@@ -326,6 +341,13 @@ int main(int argc, char **argv) {
     row("empty kernel (what a launch costs by itself)", 0.0, [&] { empty_kernel<<<1, 32>>>(); });
     const unsigned g512 = (unsigned)((n / 4 + 511) / 512), g256x8 = (unsigned)((n / 8 + 255) / 256);
     row("flat stream, 128-bit, default caching, one group per thread", bytes_all, [&] { flat128_kernel<0><<<g512, 512>>>(g, e, m, n, eta, mu); });
+    for (int per_sm : {3, 2, 1}) {                     // fewer resident CTAs: dynamic shared memory nobody uses caps them
+        char name[112];
+        snprintf(name, sizeof(name), "flat stream, 128-bit, at most %d CTAs of 512 per SM (instead of 4)", per_sm);
+        const int smem = per_sm == 3 ? 60 * 1024 : per_sm == 2 ? 90 * 1024 : 120 * 1024;
+        CHECK(cudaFuncSetAttribute(flat128_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        row(name, bytes_all, [&] { flat128_kernel<0><<<g512, 512, smem>>>(g, e, m, n, eta, mu); });
+    }
     row("flat stream, 128-bit, ld.cs / st.cs", bytes_all, [&] { flat128_kernel<1><<<g512, 512>>>(g, e, m, n, eta, mu); });
     row("flat stream, 256-bit accesses", bytes_all, [&] { flat256_kernel<<<g256x8, 256>>>(g, e, m, n, eta, mu); });
     for (int per_sm : {2, 4}) {
@@ -342,8 +364,27 @@ int main(int argc, char **argv) {
     }
     row("1-D bulk async copies through shared memory (16 KB chunks)", bytes_all,
         [&] { bulk_kernel<<<(unsigned)((n + kBulkFloats - 1) / kBulkFloats), kBulkThreads, 3 * kBulkFloats * 4>>>(g, e, m, n, eta, mu, gave_up); });
-    row("library stream kernel as shipped (grid over the tiles outside the block only)", bytes_stream,
-        [&] { defk::def_step_stream_kernel<true, 0, false, defk::kOrderRows, 2><<<stream_grid, 512>>>(a); });
+    row("library stream kernel as shipped (tiles outside the block only, CTAs of 1024 threads)", bytes_stream,
+        [&] { defk::def_step_stream_kernel<true, 0, false, defk::kOrderRows, 4><<<stream_grid, 1024>>>(a); });
+    {   // CTA size x resident CTAs, for the library kernel (prologue per CTA) and for the host-plan kernel (none)
+        const int64_t stream_tiles = tiles - tt.a_count - tt.b_count;
+#define LIB_SHAPE(T, P) { auto k_ = defk::def_step_stream_kernel<true, 0, false, defk::kOrderRows, T>; \
+        const int threads_ = 256 * T; int smem_ = 0; if (P < 2048 / threads_) smem_ = (227 * 1024 / (P + 1) + 1024) / 1024 * 1024; \
+        if (smem_) CHECK(cudaFuncSetAttribute(k_, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_)); \
+        char name_[128]; snprintf(name_, sizeof(name_), "library stream kernel, CTAs of %d threads, %d per SM", threads_, P); \
+        const dim3 grid_((unsigned)((stream_tiles + T - 1) / T), (unsigned)W); \
+        row(name_, bytes_stream, [&] { k_<<<grid_, threads_, smem_>>>(a); }); }
+#define HOST_SHAPE(T, P) { auto k_ = stream_hostplan_kernel<T>; \
+        const int threads_ = 256 * T; int smem_ = 0; if (P < 2048 / threads_) smem_ = (227 * 1024 / (P + 1) + 1024) / 1024 * 1024; \
+        if (smem_) CHECK(cudaFuncSetAttribute(k_, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_)); \
+        char name_[128]; snprintf(name_, sizeof(name_), "stream kernel with the tile plan from the host (no prologue), CTAs of %d threads, %d per SM", threads_, P); \
+        const dim3 grid_((unsigned)((stream_tiles + T - 1) / T), (unsigned)W); \
+        row(name_, bytes_stream, [&] { k_<<<grid_, threads_, smem_>>>(a, tt); }); }
+        LIB_SHAPE(1, 8) LIB_SHAPE(1, 7) LIB_SHAPE(1, 6) LIB_SHAPE(2, 4) LIB_SHAPE(2, 3) LIB_SHAPE(3, 2) LIB_SHAPE(4, 2)
+        HOST_SHAPE(1, 8) HOST_SHAPE(1, 7) HOST_SHAPE(1, 6) HOST_SHAPE(1, 5) HOST_SHAPE(2, 4) HOST_SHAPE(2, 3) HOST_SHAPE(3, 2) HOST_SHAPE(4, 2) HOST_SHAPE(4, 1)
+#undef LIB_SHAPE
+#undef HOST_SHAPE
+    }
     row("stream kernel over all tiles, block start per CTA, then loads", bytes_stream,
         [&] { stream_variant_kernel<0><<<pair_grid, 512>>>(a, s0); });
     row("stream kernel over all tiles, loads issued before the block start is known", bytes_stream,

@@ -582,6 +582,20 @@ int check_view(const def_ctx *ctx, int64_t n, int64_t ld) {
     return DEF_OK;
 }
 
+// Grid of the partial-sums kernel of def_stats: one CTA per 256 coordinate groups while that stays
+// within the scratch (kStatsMaxCtas slots); beyond, a whole number of waves of resident CTAs
+// (three of 256 threads per SM at its 64-80 registers), so that the tile-stride loop gives every
+// SM the same work and there is no ragged last wave.
+int64_t stats_grid(int64_t groups, int sm_count) {
+    int64_t ctas = (groups + defk::kStatsThreads - 1) / defk::kStatsThreads;
+    if (ctas > defk::kStatsMaxCtas) {
+        const int64_t wave = (int64_t)(sm_count > 0 ? sm_count : 1) * 3;
+        ctas = defk::kStatsMaxCtas / wave * wave;
+        if (ctas < 1) ctas = defk::kStatsMaxCtas;
+    }
+    return ctas < 1 ? 1 : ctas;
+}
+
 int width_of(int64_t ld, const void *a, const void *b, const void *c) {
     const uintptr_t bits = (uintptr_t)a | (uintptr_t)b | (uintptr_t)c;
     if ((bits & 15u) == 0 && ld % 4 == 0) return 4;
@@ -660,9 +674,7 @@ int def_stats(def_ctx *ctx, int64_t n, int64_t ld, const float *errors, double *
     }
     const int V = width_of(ld, errors, nullptr, nullptr);
     const int64_t groups = (n + V - 1) / V;
-    int64_t ctas = (groups + defk::kStatsThreads - 1) / defk::kStatsThreads;
-    if (ctas > defk::kStatsMaxCtas) ctas = defk::kStatsMaxCtas;
-    if (ctas < 1) ctas = 1;
+    const int64_t ctas = stats_grid(groups, ctx->sm_count);
     double *scratch = ctx->stats_scratch;
     if (V == 4) defk::def_stats_partial_kernel<4, 8><<<(unsigned)ctas, defk::kStatsThreads, 0, ctx->stream>>>(errors, n, ld, ctx->W, scratch);
     else if (V == 2) defk::def_stats_partial_kernel<2, 8><<<(unsigned)ctas, defk::kStatsThreads, 0, ctx->stream>>>(errors, n, ld, ctx->W, scratch);
@@ -935,9 +947,10 @@ namespace {
 constexpr int kMaxKnownDevices = 64;
 std::mutex g_static_mutex;
 double *g_static_scratch_ptr[kMaxKnownDevices] = {};
+int g_static_sm_count[kMaxKnownDevices] = {};
 
 // Device address of the static scratch on the current device (looked up on first use).
-int static_scratch_address(double **ptr_out) {
+int static_scratch_address(double **ptr_out, int *sm_count_out) {
     int dev = -1;
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) {
@@ -956,8 +969,10 @@ int static_scratch_address(double **ptr_out) {
         err = cudaGetSymbolAddress(&p, g_stats_static_scratch);
         if (err != cudaSuccess || !p) { cudaGetLastError(); return cuda_fail(err, "cudaGetSymbolAddress(static scratch)"); }
         g_static_scratch_ptr[dev] = static_cast<double *>(p);
+        g_static_sm_count[dev] = prop.multiProcessorCount;
     }
     *ptr_out = g_static_scratch_ptr[dev];
+    *sm_count_out = g_static_sm_count[dev];
     return DEF_OK;
 }
 
@@ -976,13 +991,12 @@ extern "C" int def_stats_static(const float *errors, int64_t n, int64_t ld, int3
     if (ld < n) return fail(DEF_ERR_ARG, "row stride ld=%lld is smaller than n=%lld", (long long)ld, (long long)n);
     if (!(lambda >= 0.f && lambda <= 1.f)) return fail(DEF_ERR_ARG, "lambda must be in [0, 1]");
     double *scratch = nullptr;
-    int rc = static_scratch_address(&scratch);
+    int sm_count = 0;
+    int rc = static_scratch_address(&scratch, &sm_count);
     if (rc != DEF_OK) return rc;
     const int V = width_of(ld, errors, nullptr, nullptr);
     const int64_t groups = (n + V - 1) / V;
-    int64_t ctas = (groups + defk::kStatsThreads - 1) / defk::kStatsThreads;
-    if (ctas > DEF_STATS_STATIC_SLOTS) ctas = DEF_STATS_STATIC_SLOTS;
-    if (ctas < 1) ctas = 1;
+    const int64_t ctas = stats_grid(groups, sm_count);
     if ((size_t)ctas * 2 * sizeof(double) > sizeof(double) * 2 * DEF_STATS_STATIC_SLOTS)
         return fail(DEF_ERR_ARG, "the static scratch cannot hold %lld partial sums", (long long)ctas);
     cudaStream_t stream = (cudaStream_t)cuda_stream;

@@ -478,6 +478,28 @@ __device__ __forceinline__ void flat_group_by_floats(const StepArgs &a, int64_t 
     }
 }
 
+// How many of the local coordinates [lo, hi) are block coordinates (runs A and B of touched_tiles,
+// in local coordinates).
+__device__ __forceinline__ int64_t block_coordinates_in(const StepArgs &a, int64_t s, int64_t lo, int64_t hi) {
+    const int64_t end = a.j0 + a.n;
+    int64_t a0 = (s > a.j0 ? s : a.j0) - a.j0;
+    int64_t a1 = s + a.k < a.d ? s + a.k : a.d;
+    a1 = (a1 < end ? a1 : end) - a.j0;
+    int64_t b1 = s + a.k - a.d;
+    b1 = (b1 < end ? b1 : end) - a.j0;
+    int64_t count = 0;
+    const int64_t al = lo > a0 ? lo : a0, ah = hi < a1 ? hi : a1;
+    if (ah > al) count += ah - al;
+    const int64_t bh = hi < b1 ? hi : b1;
+    if (bh > lo) count += bh - lo;
+    return count;
+}
+
+// One thread of the CTA draws the block start and sorts the CTA's kFlatTile floats into one of
+// three kinds: none of them a block coordinate's (nearly every CTA: a plain 16-byte stream with no
+// per-thread bookkeeping), all of them (nothing to do), or mixed (every float checked).
+constexpr int kFlatPlain = 0, kFlatMixed = 1, kFlatIdle = 2;
+
 template <bool MOM, int POL>
 __global__ void __launch_bounds__(kFlatThreads)
 def_step_flat_kernel(const StepArgs a) {
@@ -485,16 +507,36 @@ def_step_flat_kernel(const StepArgs a) {
     const int64_t total = (int64_t)a.W * a.n;                 // rows are contiguous: ld == n
     const int64_t base = (int64_t)blockIdx.x * kFlatTile;
     const int64_t f = base + (int64_t)threadIdx.x * 4;
-    const bool whole = f + 4 <= total;
     if (threadIdx.x == 0) {
-        shared[0] = block_start(a.seed, a.step, a.d);
-        shared[1] = base / a.n;                               // worker of the CTA's first float
-        shared[2] = base - shared[1] * a.n;                   // and its coordinate
+        const int64_t s = block_start(a.seed, a.step, a.d);
+        const int64_t w0 = base / a.n;                        // worker of the CTA's first float
+        const int64_t c0 = base - w0 * a.n;                   // and its coordinate
+        int64_t kind = kFlatMixed;
+        if (base + kFlatTile <= total) {                      // (the last, ragged CTA stays mixed)
+            // the CTA's floats are coordinates [c0, c0 + kFlatTile) of one row, or -- n >= kFlatTile --
+            // [c0, n) of one row and [0, c0 + kFlatTile - n) of the next
+            const int64_t end = c0 + kFlatTile;
+            int64_t inside = block_coordinates_in(a, s, c0, end < a.n ? end : a.n);
+            if (end > a.n) inside += block_coordinates_in(a, s, 0, end - a.n);
+            kind = inside == 0 ? kFlatPlain : inside == kFlatTile ? kFlatIdle : kFlatMixed;
+        }
+        shared[0] = s; shared[1] = c0; shared[2] = kind;
     }
     __syncthreads();
-    const int64_t s = shared[0];
-    if (f < total) {
-        int64_t c = shared[2] + (int64_t)threadIdx.x * 4;    // < 2 n because n >= kFlatTile
+    const int64_t kind = shared[2];
+    if (kind == kFlatPlain) {
+        const bool none[4] = {false, false, false, false};
+        float unused[4];
+        const Vec<4> g = load_vec<4, POL>(a.g + f);
+        const Vec<4> e = load_vec<4, POL>(a.e + f);
+        Vec<4> m, m_new, e_new;
+        if (MOM) m = load_vec<4, POL>(a.m + f);
+        worker_row<4, MOM>(g, m, e, none, a.eta, a.mu, true, m_new, e_new, unused);
+        if (MOM) store_vec<4, POL>(a.m + f, m_new);
+        store_vec<4, POL>(a.e + f, e_new);
+    } else if (kind == kFlatMixed && f < total) {
+        const int64_t s = shared[0];
+        int64_t c = shared[1] + (int64_t)threadIdx.x * 4;    // < 2 n because n >= kFlatTile
         if (c >= a.n) c -= a.n;
         bool in[4];
         bool any = false, all = true;
@@ -508,7 +550,7 @@ def_step_flat_kernel(const StepArgs a) {
             any |= in[i];
             all &= in[i];
         }
-        if (!any && whole) {
+        if (!any && f + 4 <= total) {
             const bool none[4] = {false, false, false, false};
             float unused[4];
             const Vec<4> g = load_vec<4, POL>(a.g + f);

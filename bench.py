@@ -43,8 +43,8 @@ FALLBACK_HBM_GBS = 6650.0
 # (dram__bytes_read.sum + dram__bytes_write.sum), as bytes per gradient element, and the
 # hash of the kernel source the capture was taken on.  Reported only while the source is
 # unchanged (see profiles/).
-NCU_TRAFFIC_BYTES_PER_ELEMENT = 19.42
-NCU_TRAFFIC_KERNEL_SHA256 = "deb13c2113f9bab04b32bee152010e98657aa46f3d5ca502d764c15853436536"
+NCU_TRAFFIC_BYTES_PER_ELEMENT = 19.43
+NCU_TRAFFIC_KERNEL_SHA256 = "4962b199d50a0441e2b1a5ecd45001ecf667826a029e4595b63222de7fa5d4d9"
 
 
 def _measured_peak():
@@ -155,12 +155,14 @@ def _max_over_ranks(dist, value):
     return float(t.item())
 
 
-def time_steps(B, ctx, shard, tensors, steps, warmup, seed, dist=None, flush=None, sample_clocks=None, step_fn=None):
+def time_steps(B, ctx, shard, tensors, steps, warmup, seed, dist=None, flush=None, sample_clocks=None, step_fn=None,
+               per_step_events=True):
     """Device time of `steps` steps, from CUDA events on the stream the steps are enqueued on.
     Without `flush`: an event before the first step and one after every step, launches back to
-    back (the total is first event to last).  With `flush` (a buffer larger than the L2 that is
-    rewritten between iterations): one event pair per step, summed.  Returns (total ms, max over
-    ranks; launches; this rank's per-step ms)."""
+    back (the total is first event to last); with per_step_events off, one pair around the whole
+    loop (an event between steps of a few microseconds would cost as much as the step).  With
+    `flush` (a buffer larger than the L2 that is rewritten between iterations): one event pair per
+    step, summed.  Returns (total ms, max over ranks; launches; this rank's per-step ms or None)."""
     import torch
     j0, n, ld = shard
     x, g, e, m = tensors
@@ -173,7 +175,16 @@ def time_steps(B, ctx, shard, tensors, steps, warmup, seed, dist=None, flush=Non
     launches0 = B.def_launch_count(ctx)
     if sample_clocks is not None:
         sample_clocks.start()
-    if flush is None:
+    if flush is None and not per_step_events:
+        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        start.record()
+        for t in range(steps):
+            step_fn(warmup + t)
+        end.record()
+        torch.cuda.synchronize()
+        ms = start.elapsed_time(end)
+        per_step = None
+    elif flush is None:
         marks = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
         marks[0].record()
         for t in range(steps):
@@ -201,6 +212,8 @@ def time_steps(B, ctx, shard, tensors, steps, warmup, seed, dist=None, flush=Non
 
 def step_spread(per_step):
     """Median and minimum of the per-step device times (this rank's)."""
+    if not per_step:
+        return {}
     return {"ms_per_step_median": statistics.median(per_step), "ms_per_step_min": min(per_step)}
 
 
@@ -353,7 +366,8 @@ def bench_workload(B, WL, wl, steps, warmup, dist, world, rank, sampler=None, fl
         m = None
     col_sigma = WL.column_sigma(wl, dev) if wl.grad == "per_tensor" else None
     g = WL.gradients(wl, rank, dev, col_sigma=col_sigma)   # one gradient buffer, reused: values do not steer the kernel
-    ms, launches, per_step = time_steps(B, ctx, (j0, n, n), (x, g, e, m), steps, warmup, wl.rbgs_seed, dist, flush, sampler)
+    ms, launches, per_step = time_steps(B, ctx, (j0, n, n), (x, g, e, m), steps, warmup, wl.rbgs_seed, dist, flush, sampler,
+                                        per_step_events=wl.algorithmic_bytes_per_step() >= 1e9)
     per_el = 20 if wl.momentum != 0.0 else 12
     alg_bytes = per_el * wl.W * n + 8 * k_global / world
     kernels = None

@@ -380,6 +380,42 @@ def bench_workload(B, WL, wl, steps, warmup, dist, world, rank, sampler=None, fl
     return ms, launches, wl.W * d_global, alg_bytes, kernels, per_step
 
 
+def bench_graph_replay(B, WL, wl, replays=5):
+    """The workload's whole loop of steps (each with its own step number) recorded once into a CUDA
+    graph and replayed: what a launch-bound tiny model costs per step when the host is out of the way."""
+    import torch
+    dev = torch.device("cuda")
+    ctx = B.def_create(wl.d, wl.W, wl.k, wl.variant, wl.lr, wl.momentum, (wl.lam, 0.0))
+    x = WL.initial_params(wl, dev)
+    e, m = WL.zeros_state(wl, dev)
+    if wl.momentum == 0.0:
+        m = None
+    g = WL.gradients(wl, 0, dev)
+    B.def_step(ctx, x, g, e, m, 0, wl.rbgs_seed)            # the first call (device query) stays outside the capture
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        B.def_set_stream(ctx, side)
+        with torch.cuda.graph(graph, stream=side):
+            for t in range(wl.steps):
+                B.def_step(ctx, x, g, e, m, t, wl.rbgs_seed)
+        B.def_set_stream(ctx, None)
+    graph.replay()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(replays):
+        graph.replay()
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / (replays * wl.steps)
+    B.def_destroy(ctx)
+    del graph, x, g, e, m
+    torch.cuda.empty_cache()
+    return ms
+
+
 def bench_aux(B, WL, wl, reps=5):
     """Device time of the helpers around the step on the same workload: the detach point
     (Algorithm 1's detach step), DEF's returned model and the distances of Eq. 9."""
@@ -727,7 +763,9 @@ def main():
                     ms_r, _, _, _, _, per_r = bench_workload(B, WL, w, w.steps, 3, None, 1, 0, flush=None)
                     resident = {"ms_per_step": ms_r / w.steps, **step_spread(per_r),
                                 "effective_GB/s": bytes_w * w.steps / (ms_r * 1e-3) / 1e9,
-                                "note": "state stays in the 126 MB L2 between steps: not an HBM figure"}
+                                "graph_replay_ms_per_step": bench_graph_replay(B, WL, w),
+                                "note": "state stays in the 126 MB L2 between steps: not an HBM figure; graph_replay = the "
+                                        "loop of steps recorded into one CUDA graph and replayed"}
                 per.append({"cfg": w.cfg, "name": w.name, "ratio": w.ratio, "variant": WL.VARIANT_NAMES[w.variant],
                             "steps": w.steps, "ms_per_step": ms_w / w.steps, **step_spread(per_w),
                             "elements_per_s": el_w * w.steps / (ms_w * 1e-3),

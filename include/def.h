@@ -304,9 +304,10 @@ int def_set_small_step_bytes(def_ctx *ctx, int64_t bytes);
 /*
  * Whether the second kernel of a pair may start while the first (the tiles that touch the block)
  * is still running -- they write disjoint floats, and work enqueued after the pair is ordered
- * behind both either way.  DEF_OVERLAP_AUTO (default) lets the library decide from the sizes,
- * DEF_OVERLAP_NEVER runs the two one after the other, DEF_OVERLAP_ALWAYS side by side.
- * Results are bit-identical in every mode.
+ * behind both either way.  DEF_OVERLAP_AUTO (default) leaves the choice to the library (side by
+ * side at every size: it was at least as fast wherever it was measured), DEF_OVERLAP_NEVER runs
+ * the two one after the other, DEF_OVERLAP_ALWAYS side by side.  Results are bit-identical in
+ * every mode.
  */
 enum { DEF_OVERLAP_AUTO = 0, DEF_OVERLAP_NEVER = 1, DEF_OVERLAP_ALWAYS = 2 };
 int def_set_pair_overlap(def_ctx *ctx, int32_t mode);

@@ -182,17 +182,13 @@ cudaError_t counted_launch(def_ctx *ctx, int kind, cudaStream_t stream, Launch l
 // Launch of the stream kernel right after the block kernel of the same step.  The two work on
 // disjoint tiles, so the stream kernel is allowed to start while the block kernel still runs
 // (programmatic stream serialization; the block kernel releases its dependents at once).  That
-// hides the block kernel's latency-bound run on mid-sized models.  The stream kernel's threads
-// end with a wait for the block kernel's grid, so whatever is enqueued later, being ordered
-// behind the stream kernel, is ordered behind both.  Not used in timing mode, where each
-// kernel is measured alone, nor when the block kernel went to another stream (`beside` false:
-// the two then overlap as work on two streams does).
-bool overlap_allowed(const def_ctx *ctx, const defk::StepArgs &a) {
-    (void)a;
-    if (ctx->pair_overlap == DEF_OVERLAP_NEVER) return false;
-    return true;
-}
-
+// hides the block kernel's latency-bound run on small and mid-sized models.  One thread of the
+// stream kernel ends with a wait for the block kernel's grid, so whatever is enqueued later, being
+// ordered behind the stream kernel, is ordered behind both.  Not used in timing mode, where each
+// kernel is measured alone, under DEF_OVERLAP_NEVER, nor when the block kernel went to another
+// stream (`beside` false: the two then overlap as work on two streams does).  DEF_OVERLAP_AUTO
+// overlaps at every size: side by side was at least as fast as one after the other wherever it
+// was measured (1 MB to 44 GB per step, k from d/1000 to d/8).
 template <typename Kernel>
 cudaError_t launch_beside_block_kernel(const def_ctx *ctx, Kernel kernel, dim3 grid, unsigned threads,
                                        cudaStream_t stream, const defk::StepArgs &a, bool beside = true) {
@@ -202,7 +198,8 @@ cudaError_t launch_beside_block_kernel(const def_ctx *ctx, Kernel kernel, dim3 g
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = (ctx->timing || !beside || !overlap_allowed(ctx, a)) ? 0 : 1;
+    attr[0].val.programmaticStreamSerializationAllowed =
+        (ctx->timing || !beside || ctx->pair_overlap == DEF_OVERLAP_NEVER) ? 0 : 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, a);
@@ -217,12 +214,12 @@ cudaError_t launch_beside_block_kernel(const def_ctx *ctx, Kernel kernel, dim3 g
 constexpr int kDetachChunkCtas = 256;
 
 // Steps that move fewer bytes than this run as ONE launch of the general kernel instead of the
-// kernel pair.  With the stream kernel allowed to start beside the block kernel the pair is at
-// least as fast from cold memory at every size measured (flushed L2: 13.3 vs 14.3 us at 40 MB,
-// 19.5 vs 20.4 us at 80 MB, 27.6 vs 28.7 us on the 137 MB ResNet-56-sized workload, 275 vs 287 us
-// at 1.9 GB); only tiny models stepped back to back out of the L2 are bound by the launches
-// themselves and prefer one (7.4 vs 9.4 us at 40 MB, 10.4 vs 10.8 us at 80 MB; the pair leads
-// from 160 MB).  Hence 128 MiB.
+// kernel pair.  From cold caches (L2 flushed before every step) the single launch is 1 us ahead up
+// to about 20 MB (8.2 vs 9.2 us at 1-5 MB, 10.2 vs 11.3 at 21 MB), level at 80 MB (19.4 us both)
+// and behind from the 137 MB ResNet-56-sized workload on (28.7 vs 27.6 us; 55.3 vs 54.3 at
+// 320 MB); stepped back to back out of the L2, where the launches themselves are the bound, it
+// leads up to 137 MB (6.2 vs 8.2 us at 1 MB, 10.4 vs 10.5 at 80 MB, 14.6 vs 16.4 at 137 MB) and
+// trails from 320 MB (52.7 vs 49.5 us).  Hence 128 MiB.
 // def_set_small_step_bytes changes it per context.
 constexpr int64_t kSmallStepBytesDefault = (int64_t)128 << 20;
 

@@ -97,3 +97,27 @@ def test_pair_back_to_back_with_detach_output(B):
     for w in range(W):
         assert np.array_equal(zh[w], oracle.detach(xo, np.ascontiguousarray(eo[w]), lam)), w
     B.def_destroy(ctx)
+
+
+@pytest.mark.parametrize("mode", ["never", "always"])
+def test_pair_overlap_modes_give_the_same_bits(B, mode):
+    """The second kernel of the pair started beside the first, or strictly after it: same results."""
+    dev = torch.device("cuda")
+    d, W, k, seed, lr, mu = 700_000, 6, 200_000, 9, 0.1, 0.9
+    rng = np.random.default_rng(17)
+    gh = (0.1 * rng.standard_normal((W, d))).astype(np.float32)
+    g = torch.from_numpy(gh).to(dev)
+    x = torch.from_numpy((0.05 * rng.standard_normal(d)).astype(np.float32)).to(dev)
+    e = torch.zeros(W, d, device=dev); m = torch.zeros(W, d, device=dev)
+    xo = x.cpu().numpy().copy(); eo = np.zeros((W, d), np.float32); mo = np.zeros((W, d), np.float32)
+    ctx = B.def_create(d, W, k, B.DEF_VARIANT_DEF, lr, mu)
+    B.def_set_small_step_bytes(ctx, 0)
+    B.def_set_pair_overlap(ctx, B.DEF_OVERLAP_NEVER if mode == "never" else B.DEF_OVERLAP_ALWAYS)
+    for t in range(8):
+        B.def_step(ctx, x, g, e, m, t, seed)
+    torch.cuda.synchronize()
+    for t in range(8):
+        oracle.step(xo, gh, eo, mo, d=d, k=k, s=oracle.block_start(seed, t, d), eta=lr, mu=mu)
+    assert np.array_equal(x.cpu().numpy(), xo) and np.array_equal(e.cpu().numpy(), eo) and np.array_equal(m.cpu().numpy(), mo)
+    assert B.lib.def_set_pair_overlap(ctx.handle, 7) == B.DEF_ERR_ARG
+    B.def_destroy(ctx)

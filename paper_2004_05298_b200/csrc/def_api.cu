@@ -593,6 +593,32 @@ int64_t stats_grid(int64_t groups, int sm_count) {
     return ctas < 1 ? 1 : ctas;
 }
 
+// The two kernels of def_stats / def_stats_static: per-CTA partial sums into `scratch`, then one
+// CTA that adds them.  The second is launched with programmatic stream serialization: it is set
+// up while the first runs and waits (griddepcontrol.wait) for that grid to complete before it
+// reads a partial sum, which takes its launch latency out of the call.
+int launch_stats(const float *errors, int64_t n, int64_t ld, int W, float lambda, int V, int64_t ctas,
+                 double *scratch, double *stats_out, cudaStream_t stream) {
+    if (V == 4) defk::def_stats_partial_kernel<4, 8><<<(unsigned)ctas, defk::kStatsThreads, 0, stream>>>(errors, n, ld, W, scratch);
+    else if (V == 2) defk::def_stats_partial_kernel<2, 8><<<(unsigned)ctas, defk::kStatsThreads, 0, stream>>>(errors, n, ld, W, scratch);
+    else defk::def_stats_partial_kernel<1, 8><<<(unsigned)ctas, defk::kStatsThreads, 0, stream>>>(errors, n, ld, W, scratch);
+    cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) return cuda_fail(err, "def_stats kernel launch");
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(1);
+    cfg.blockDim = dim3(defk::kStatsThreads);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    err = cudaLaunchKernelEx(&cfg, defk::def_stats_final_kernel, (const double *)scratch, (int)ctas, W, lambda, stats_out);
+    if (err == cudaSuccess) err = cudaGetLastError();
+    if (err != cudaSuccess) return cuda_fail(err, "def_stats final kernel launch");
+    return DEF_OK;
+}
+
 int width_of(int64_t ld, const void *a, const void *b, const void *c) {
     const uintptr_t bits = (uintptr_t)a | (uintptr_t)b | (uintptr_t)c;
     if ((bits & 15u) == 0 && ld % 4 == 0) return 4;
@@ -672,17 +698,9 @@ int def_stats(def_ctx *ctx, int64_t n, int64_t ld, const float *errors, double *
     const int V = width_of(ld, errors, nullptr, nullptr);
     const int64_t groups = (n + V - 1) / V;
     const int64_t ctas = stats_grid(groups, ctx->sm_count);
-    double *scratch = ctx->stats_scratch;
-    if (V == 4) defk::def_stats_partial_kernel<4, 8><<<(unsigned)ctas, defk::kStatsThreads, 0, ctx->stream>>>(errors, n, ld, ctx->W, scratch);
-    else if (V == 2) defk::def_stats_partial_kernel<2, 8><<<(unsigned)ctas, defk::kStatsThreads, 0, ctx->stream>>>(errors, n, ld, ctx->W, scratch);
-    else defk::def_stats_partial_kernel<1, 8><<<(unsigned)ctas, defk::kStatsThreads, 0, ctx->stream>>>(errors, n, ld, ctx->W, scratch);
-    cudaError_t err = cudaGetLastError();
-    if (err != cudaSuccess) return cuda_fail(err, "def_stats kernel launch");
-    defk::def_stats_final_kernel<<<1, defk::kStatsThreads, 0, ctx->stream>>>(scratch, (int)ctas, ctx->W, ctx->lambda, stats_out);
-    err = cudaGetLastError();
-    if (err != cudaSuccess) return cuda_fail(err, "def_stats final kernel launch");
-    ctx->launches += 2;
-    return DEF_OK;
+    rc = launch_stats(errors, n, ld, ctx->W, ctx->lambda, V, ctas, ctx->stats_scratch, stats_out, ctx->stream);
+    if (rc == DEF_OK) ctx->launches += 2;
+    return rc;
 }
 
 int def_step_columns(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, float *params,
@@ -996,16 +1014,7 @@ extern "C" int def_stats_static(const float *errors, int64_t n, int64_t ld, int3
     const int64_t ctas = stats_grid(groups, sm_count);
     if ((size_t)ctas * 2 * sizeof(double) > sizeof(double) * 2 * DEF_STATS_STATIC_SLOTS)
         return fail(DEF_ERR_ARG, "the static scratch cannot hold %lld partial sums", (long long)ctas);
-    cudaStream_t stream = (cudaStream_t)cuda_stream;
     // Every slot the second kernel reads ([0, ctas)) is written by the first in this same call,
     // so nothing left over from an earlier call is ever read and nothing needs clearing.
-    if (V == 4) defk::def_stats_partial_kernel<4, 8><<<(unsigned)ctas, defk::kStatsThreads, 0, stream>>>(errors, n, ld, W, scratch);
-    else if (V == 2) defk::def_stats_partial_kernel<2, 8><<<(unsigned)ctas, defk::kStatsThreads, 0, stream>>>(errors, n, ld, W, scratch);
-    else defk::def_stats_partial_kernel<1, 8><<<(unsigned)ctas, defk::kStatsThreads, 0, stream>>>(errors, n, ld, W, scratch);
-    cudaError_t err = cudaGetLastError();
-    if (err != cudaSuccess) return cuda_fail(err, "def_stats_static kernel launch");
-    defk::def_stats_final_kernel<<<1, defk::kStatsThreads, 0, stream>>>(scratch, (int)ctas, W, lambda, stats_out);
-    err = cudaGetLastError();
-    if (err != cudaSuccess) return cuda_fail(err, "def_stats_static final kernel launch");
-    return DEF_OK;
+    return launch_stats(errors, n, ld, W, lambda, V, ctas, scratch, stats_out, (cudaStream_t)cuda_stream);
 }

@@ -108,6 +108,9 @@ __global__ void __launch_bounds__(kStatsThreads)
 def_stats_partial_kernel(const float *__restrict__ e, int64_t n, int64_t ld, int W,
                          double *__restrict__ scratch) {
     __shared__ double smem[kStatsThreads / 32];
+    // the one-CTA kernel that adds the partial sums may be set up while this grid runs (it waits
+    // for this grid before it reads anything); a no-op when it was launched the ordinary way
+    release_dependent_grids();
     double sq = 0.0, mean_sq = 0.0;
     const double inv_W = 1.0 / (double)W;
     const int64_t groups = (n + V - 1) / V;
@@ -160,13 +163,13 @@ def_stats_partial_kernel(const float *__restrict__ e, int64_t n, int64_t ld, int
 }
 
 __global__ void __launch_bounds__(kStatsThreads)
-def_stats_final_kernel(const double *__restrict__ scratch, int ctas, int W, float lambda,
-                       double *__restrict__ out) {
+def_stats_final_kernel(const double *scratch, int ctas, int W, float lambda, double *out) {
     __shared__ double smem[kStatsThreads / 32];
+    grid_dependency_wait();                     // the partial sums are complete and visible from here on
     double sq = 0.0, mean_sq = 0.0;
     for (int i = threadIdx.x; i < ctas; i += blockDim.x) {
-        sq += scratch[2 * i];
-        mean_sq += scratch[2 * i + 1];
+        sq += __ldcg(scratch + 2 * i);          // from the L2, where the other grid's stores are
+        mean_sq += __ldcg(scratch + 2 * i + 1);
     }
     const double sq_all = cta_sum(sq, smem);
     const double mean_all = cta_sum(mean_sq, smem);

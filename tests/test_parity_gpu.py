@@ -405,10 +405,14 @@ def test_config5_full_size_sampled(B, ratio, variant):
 # ---------------------------------------------------------------------------
 # column ranges, host memory, streams, resume
 # ---------------------------------------------------------------------------
+@pytest.mark.parametrize("ratio", [32, 2], ids=["k=d/32", "k=d/2"])
 @pytest.mark.parametrize("pair", [True, False], ids=["pair", "general"])
-def test_step_columns_equals_whole_step(B, pair):
+def test_step_columns_equals_whole_step(B, pair, ratio):
+    """Column ranges of the model stepped separately (aligned and unaligned cuts, padded rows) against
+    the whole step, on steps whose block lies inside a range, straddles cuts, and wraps past d: every
+    range has to find its own share of the block's tiles."""
     dev = torch.device("cuda")
-    wl = WL.get(2).scaled(200_001, W=6)
+    wl = WL.get(2).scaled(200_001, W=6).with_ratio(ratio)
     d, W, k = wl.d, wl.W, wl.k
     x = WL.initial_params(wl, dev); e, m = WL.zeros_state(wl, dev)
     cuts = [0, 4, 70_000, 70_003, 150_002, d]                     # aligned and unaligned pieces
@@ -417,7 +421,8 @@ def test_step_columns_equals_whole_step(B, pair):
     B.def_set_small_step_bytes(ctx, 0 if pair else 1 << 60)
     es = [torch.zeros(W, b - a + 5, device=dev) for a, b in zip(cuts[:-1], cuts[1:])]   # ld = n + 5
     ms = [torch.zeros(W, b - a + 5, device=dev) for a, b in zip(cuts[:-1], cuts[1:])]
-    for t in range(6):
+    steps = sorted(set(list(range(5)) + find_steps(d, k, 9, lambda s: s + k > d) + find_steps(d, k, 9, lambda s: s < 70_000 < s + k)))
+    for t in steps:
         g = WL.gradients(wl, t, dev)
         B.def_step(ctx, x, g, e, m, t, 9)
         for i, (a, b) in enumerate(zip(cuts[:-1], cuts[1:])):
@@ -428,6 +433,42 @@ def test_step_columns_equals_whole_step(B, pair):
         assert torch.equal(xs[i], x[a:b])
         assert torch.equal(es[i][:, : b - a], e[:, a:b]) and torch.equal(ms[i][:, : b - a], m[:, a:b])
         assert not es[i][:, b - a:].any() and not ms[i][:, b - a:].any(), "padding columns were written"
+    B.def_destroy(ctx)
+
+
+@pytest.mark.parametrize("ratio", [32, 3, 1], ids=["k=d/32", "k=d/3", "k=d"])
+def test_column_shards_on_the_kernel_pair(B, ratio):
+    """Column shards with 16-byte aligned rows run the kernel pair, each kernel with a grid for its
+    own tiles of the shard only: shards that hold all, part or none of the block (one run or both,
+    the block wrapping past d into the first shard) against the oracle on every element."""
+    dev = torch.device("cuda")
+    d, W, seed, lr, mu = 600_000, 5, 21, 0.1, 0.9
+    k = max(1, d // ratio)
+    cuts = [0, 1024, 100_004, 100_008, 333_336, 599_996, d]      # multiples of 4: every shard keeps 16-byte rows
+    rng = np.random.default_rng(ratio)
+    x0 = (0.05 * rng.standard_normal(d)).astype(np.float32)
+    xo = x0.copy(); eo = np.zeros((W, d), np.float32); mo = np.zeros((W, d), np.float32)
+    ctx = B.def_create(d, W, k, 0, lr, mu)
+    B.def_set_small_step_bytes(ctx, 0)
+    B.def_set_kernel_timing(ctx, True)
+    shards = []
+    for a, b in zip(cuts[:-1], cuts[1:]):
+        n = b - a
+        shards.append((a, n, torch.from_numpy(x0[a:b].copy()).to(dev), torch.zeros(W, n, device=dev), torch.zeros(W, n, device=dev)))
+    steps = sorted(set([0, 1, 2] + find_steps(d, k, seed, lambda s: s + k > d) + find_steps(d, k, seed, lambda s: s < 100_006 < s + k)))
+    for t in steps:
+        gh = (0.1 * rng.standard_normal((W, d))).astype(np.float32)
+        oracle.step(xo, gh, eo, mo, d=d, k=k, s=oracle.block_start(seed, t, d), eta=lr, mu=mu)
+        for a, n, xs, es, ms in shards:
+            g = torch.from_numpy(np.ascontiguousarray(gh[:, a:a + n])).to(dev)
+            plan = B.def_tile_plan(ctx, a, n, t, seed)
+            assert plan[1] + plan[2] + plan[3] == -(-n // 1024)
+            B.def_step_columns(ctx, a, n, n, xs, g, es, ms, t, seed)
+    assert B.def_kernel_time(ctx, B.DEF_KERNEL_GENERAL)[1] == 0
+    assert B.def_kernel_time(ctx, B.DEF_KERNEL_STREAM)[1] == len(steps) * len(shards)
+    for a, n, xs, es, ms in shards:
+        assert np.array_equal(xs.cpu().numpy(), xo[a:a + n]), a
+        assert np.array_equal(es.cpu().numpy(), eo[:, a:a + n]) and np.array_equal(ms.cpu().numpy(), mo[:, a:a + n]), a
     B.def_destroy(ctx)
 
 

@@ -170,6 +170,8 @@ def time_steps(B, ctx, shard, tensors, steps, warmup, seed, dist=None, flush=Non
         def step_fn(t):
             B.def_step_columns(ctx, j0, n, ld, x, g, e, m, t, seed)
     for t in range(warmup):
+        if flush is not None:
+            flush.add_(1.0)                                # warm up the way the timed steps run
         step_fn(t)
     _barrier(dist)
     launches0 = B.def_launch_count(ctx)

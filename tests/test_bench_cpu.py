@@ -48,3 +48,32 @@ def test_reference_arm_prints_the_contract_line():
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2"],
                          capture_output=True, text=True, timeout=120, env=env)
     assert out.returncode == 0 and out.stdout.strip() == ""
+
+
+def test_config_names_the_sharding_that_ran():
+    bench = _bench()
+    from paper_2004_05298_b200 import workloads as WL
+    wl = WL.get(5)
+    one = bench.workload_config(wl, 1, "single")
+    rows = bench.workload_config(wl, 8, "rows")
+    cols = bench.workload_config(wl, 8, "columns")
+    assert one["W"] == 16 and one["d"] == wl.d and "no collective" in one["parallelism"]
+    assert rows["W"] == 128 and rows["d"] == wl.d and rows["k"] == wl.k          # K = 16 N workers, full model per GPU
+    assert "NCCL all-reduce" in rows["parallelism"] and "8 GPU" in rows["parallelism"]
+    assert cols["W"] == 16 and cols["d"] == 8 * wl.d and cols["k"] == 8 * wl.d // wl.ratio
+    assert all("model" not in c for c in (one, rows, cols))                       # workload keys, no model keys
+    assert "flushed" in bench.workload_config(WL.get(1), 1, "single")["l2"]
+
+
+def test_roofline_object_and_step_spread():
+    bench = _bench()
+    kernels = [{"kernel": "def_step_stream_kernel", "launches": 4, "ms_per_launch": 6.0, "algorithmic_bytes_per_launch": 42e9, "GB/s": 7000.0},
+               {"kernel": "def_step_block_kernel", "launches": 4, "ms_per_launch": 0.2, "algorithmic_bytes_per_launch": 1.4e9, "GB/s": 7000.0}]
+    r = bench.roofline_of(kernels, 6900.0, 44e9, 2.0, 6550.0, "measured")
+    assert r["bound"] == "hbm" and r["kernel"] == "def_step_stream_kernel" and r["unit"] == "GB/s"
+    assert abs(r["frac"] - 7000.0 / 6550.0) < 1e-12 and r["peak_kind"] == "of measured"
+    assert r["traffic"] is None or abs(r["traffic"] - bench.NCU_TRAFFIC_BYTES_PER_ELEMENT * 42e9 / 20.0) < 1.0
+    # the traffic figure is only reported for the kernel file it was captured on
+    assert (r["traffic"] is not None) == (bench.NCU_TRAFFIC_KERNEL_SHA256 == bench._kernel_hash())
+    assert bench.step_spread([3.0, 1.0, 2.0]) == {"ms_per_step_median": 2.0, "ms_per_step_min": 1.0}
+    assert bench.step_spread(None) == {}

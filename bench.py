@@ -39,11 +39,12 @@ METRIC = "DEF step gradient elements/s (W*d per step)"
 UNIT = "elements/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM traffic of one def_step_stream_kernel launch from an ncu capture
-# (dram__bytes_read.sum + dram__bytes_write.sum), as bytes per gradient element, and the
-# hash of the kernel source the capture was taken on.  Reported only while the source is
-# unchanged (see profiles/).
-NCU_TRAFFIC_BYTES_PER_ELEMENT = 19.43
+# DRAM traffic of one def_step_stream_kernel launch from ncu captures
+# (dram__bytes_read.sum + dram__bytes_write.sum), as bytes per gradient element, per workload:
+# config 5 from a one-pass capture of these two counters on the timed launch configuration itself,
+# config 3 from the full-set capture.  Reported only for those workloads and only while the kernel
+# source is the file the captures were taken on (hash below; see profiles/).
+NCU_TRAFFIC_BYTES_PER_ELEMENT = {5: 19.98, 3: 19.43}
 NCU_TRAFFIC_KERNEL_SHA256 = "4962b199d50a0441e2b1a5ecd45001ecf667826a029e4595b63222de7fa5d4d9"
 
 
@@ -634,14 +635,15 @@ def workload_config(wl, world, sharding):
     return cfg
 
 
-def roofline_of(kernels, step_gbs, alg_bytes, launches_per_step, peak, peak_kind):
+def roofline_of(kernels, step_gbs, alg_bytes, launches_per_step, peak, peak_kind, cfg=None):
     """The roofline object of the JSON line: the dominant kernel against the measured HBM peak."""
     top = max(kernels, key=lambda kk: kk["ms_per_launch"] * kk["launches"])
     achieved = top["GB/s"] if top["GB/s"] is not None else step_gbs
     traffic = None
-    if (NCU_TRAFFIC_BYTES_PER_ELEMENT is not None and NCU_TRAFFIC_KERNEL_SHA256 == _kernel_hash()
+    per_element = NCU_TRAFFIC_BYTES_PER_ELEMENT.get(cfg)
+    if (per_element is not None and NCU_TRAFFIC_KERNEL_SHA256 == _kernel_hash()
             and top["algorithmic_bytes_per_launch"] and top["kernel"] == "def_step_stream_kernel"):
-        traffic = NCU_TRAFFIC_BYTES_PER_ELEMENT * top["algorithmic_bytes_per_launch"] / 20.0
+        traffic = per_element * top["algorithmic_bytes_per_launch"] / 20.0
     return {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
             "traffic": traffic, "peak_kind": "of %s" % peak_kind, "frac_of_8000_nominal": achieved / 8000.0,
             "kernel": top["kernel"], "algorithmic_bytes_per_launch": top["algorithmic_bytes_per_launch"],
@@ -716,7 +718,8 @@ def main():
         step_gbs = alg_bytes * args.steps / (ms * 1e-3) / 1e9
         line.update({"value": elements * args.steps / (ms * 1e-3), "ms_per_step": ms / args.steps, **step_spread(per_step),
                      "gpu_launches": launches, "clocks": clocks,
-                     "roofline": roofline_of(kernels, step_gbs, alg_bytes, launches / args.steps, peak, peak_kind)})
+                     "roofline": roofline_of(kernels, step_gbs, alg_bytes, launches / args.steps, peak, peak_kind,
+                                            cfg=wl.cfg if wl.ratio == WL.get(wl.cfg).ratio and wl.momentum != 0.0 else None)})
         if args.aux or not args.no_extras:
             ms_z, _, _, bytes_z, _, per_z = bench_rows(B, WL, wl, min(args.steps, 10), 3, dist, world, rank, None,
                                                        side_stream=side, detach=True)
@@ -742,7 +745,8 @@ def main():
     step_gbs = alg_bytes * args.steps / (ms * 1e-3) / 1e9
     line.update({"value": elements * args.steps / (ms * 1e-3), "ms_per_step": ms / args.steps, **step_spread(per_step),
                  "gpu_launches": launches, "clocks": clocks,
-                 "roofline": roofline_of(kernels, step_gbs, alg_bytes, launches / args.steps, peak, peak_kind)})
+                 "roofline": roofline_of(kernels, step_gbs, alg_bytes, launches / args.steps, peak, peak_kind,
+                                            cfg=wl.cfg if wl.ratio == WL.get(wl.cfg).ratio and wl.momentum != 0.0 else None)})
 
     if args.no_extras and args.aux and world == 1:
         line["aux"] = bench_aux(B, WL, wl)

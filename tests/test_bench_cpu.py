@@ -69,10 +69,11 @@ def test_roofline_object_and_step_spread():
     bench = _bench()
     kernels = [{"kernel": "def_step_stream_kernel", "launches": 4, "ms_per_launch": 6.0, "algorithmic_bytes_per_launch": 42e9, "GB/s": 7000.0},
                {"kernel": "def_step_block_kernel", "launches": 4, "ms_per_launch": 0.2, "algorithmic_bytes_per_launch": 1.4e9, "GB/s": 7000.0}]
-    r = bench.roofline_of(kernels, 6900.0, 44e9, 2.0, 6550.0, "measured")
+    r = bench.roofline_of(kernels, 6900.0, 44e9, 2.0, 6550.0, "measured", cfg=5)
+    assert bench.roofline_of(kernels, 6900.0, 44e9, 2.0, 6550.0, "measured", cfg=4)["traffic"] is None   # no capture for that workload
     assert r["bound"] == "hbm" and r["kernel"] == "def_step_stream_kernel" and r["unit"] == "GB/s"
     assert abs(r["frac"] - 7000.0 / 6550.0) < 1e-12 and r["peak_kind"] == "of measured"
-    assert r["traffic"] is None or abs(r["traffic"] - bench.NCU_TRAFFIC_BYTES_PER_ELEMENT * 42e9 / 20.0) < 1.0
+    assert r["traffic"] is None or abs(r["traffic"] - bench.NCU_TRAFFIC_BYTES_PER_ELEMENT[5] * 42e9 / 20.0) < 1.0
     # the traffic figure is only reported for the kernel file it was captured on
     assert (r["traffic"] is not None) == (bench.NCU_TRAFFIC_KERNEL_SHA256 == bench._kernel_hash())
     assert bench.step_spread([3.0, 1.0, 2.0]) == {"ms_per_step_median": 2.0, "ms_per_step_min": 1.0}

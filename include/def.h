@@ -124,6 +124,8 @@ int def_step_columns(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, float *par
  * evaluates at x_{t+1} itself and has no use for it).  It costs one more [W, d] write:
  * 24 instead of 20 bytes per gradient element.  detached_out [W, ld] must overlap none of
  * the other tensors.  Other arguments and errors as for def_step / def_step_columns.
+ * Contiguous rows with d % 4 != 0 (16-byte aligned bases, params included) keep 128-bit accesses
+ * here too, 2-4 % behind rows padded to a multiple of 4 floats (ld = 4 * ceil(d / 4)).
  */
 int def_step_detach(def_ctx *ctx, float *params, const float *grads, float *errors, float *mom,
                     float *detached_out, uint64_t step, uint64_t seed);

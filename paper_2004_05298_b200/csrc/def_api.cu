@@ -311,23 +311,37 @@ int enqueue_columns(def_ctx *ctx, int64_t j0, int64_t n, int64_t ld, float *x, c
     cudaError_t err = cudaSuccess;
     // Contiguous rows that are not 16-byte aligned but whose bases are: block coordinates by one
     // kernel, everything else as a flat stream that ignores the row boundaries.
-    const bool flat_ok = V < 4 && ld == n && n >= defk::kFlatTile && !z &&
+    const bool flat_ok = V < 4 && ld == n && n >= defk::kFlatTile &&
                          ctx->compressor == DEF_COMPRESSOR_RBGS &&
-                         (((uintptr_t)g | (uintptr_t)e | (uintptr_t)m) & 15u) == 0 &&
+                         (((uintptr_t)g | (uintptr_t)e | (uintptr_t)m | (uintptr_t)z | (uintptr_t)(z ? x : nullptr)) & 15u) == 0 &&
                          20 * (int64_t)ctx->W * n >= ctx->small_step_bytes;
     if (flat_ok) {
         const int64_t block_grid = (ctx->k + 255) / 256;
-        const int64_t flat_grid = ((int64_t)ctx->W * n + defk::kFlatTile - 1) / defk::kFlatTile;
-        if (block_grid > 0x7fffffffLL || flat_grid > 0x7fffffffLL) return fail(DEF_ERR_ARG, "problem too large for one grid");
+        const int64_t flat_ctas = ((int64_t)ctx->W * n + defk::kFlatTile - 1) / defk::kFlatTile;
+        dim3 flat_grid((unsigned)flat_ctas);
+        if (z) {   // chunked order: (row, segment of coordinates) by (slot in it), so that x stays in the L2
+            const int64_t segment = n < defk::kFlatSegment ? n : defk::kFlatSegment;
+            const int64_t slots = (segment + defk::kFlatTile - 1) / defk::kFlatTile;
+            const int64_t segments = (n + defk::kFlatSegment - 1) / defk::kFlatSegment;
+            if (segments > 65535 || slots * ctx->W > 0x7fffffffLL) return fail(DEF_ERR_ARG, "problem too large for one grid");
+            a.chunk = (int32_t)slots;
+            flat_grid = dim3((unsigned)(slots * ctx->W), (unsigned)segments);
+        }
+        if (block_grid > 0x7fffffffLL || flat_ctas > 0x7fffffffLL) return fail(DEF_ERR_ARG, "problem too large for one grid");
         const bool beside = block_stream == stream;
         err = counted_launch(ctx, DEF_KERNEL_BLOCK, block_stream, [&] {
-            if (m) defk::def_step_block_columns_kernel<true, 8, kPolicy><<<(unsigned)block_grid, 256, 0, block_stream>>>(a);
-            else defk::def_step_block_columns_kernel<false, 8, kPolicy><<<(unsigned)block_grid, 256, 0, block_stream>>>(a);
+            const unsigned grid = (unsigned)block_grid;
+            if (m && z) defk::def_step_block_columns_kernel<true, 8, kPolicy, true><<<grid, 256, 0, block_stream>>>(a);
+            else if (m) defk::def_step_block_columns_kernel<true, 8, kPolicy, false><<<grid, 256, 0, block_stream>>>(a);
+            else if (z) defk::def_step_block_columns_kernel<false, 8, kPolicy, true><<<grid, 256, 0, block_stream>>>(a);
+            else defk::def_step_block_columns_kernel<false, 8, kPolicy, false><<<grid, 256, 0, block_stream>>>(a);
         });
         if (err != cudaSuccess) return cuda_fail(err, "def_step block-columns kernel launch");
         err = counted_launch(ctx, DEF_KERNEL_STREAM, stream, [&] {
-            if (m) launch_beside_block_kernel(ctx, defk::def_step_flat_kernel<true, kPolicy>, dim3((unsigned)flat_grid), defk::kFlatThreads, stream, a, beside);
-            else launch_beside_block_kernel(ctx, defk::def_step_flat_kernel<false, kPolicy>, dim3((unsigned)flat_grid), defk::kFlatThreads, stream, a, beside);
+            if (m && z) launch_beside_block_kernel(ctx, defk::def_step_flat_kernel<true, kPolicy, true>, flat_grid, defk::kFlatThreads, stream, a, beside);
+            else if (m) launch_beside_block_kernel(ctx, defk::def_step_flat_kernel<true, kPolicy, false>, flat_grid, defk::kFlatThreads, stream, a, beside);
+            else if (z) launch_beside_block_kernel(ctx, defk::def_step_flat_kernel<false, kPolicy, true>, flat_grid, defk::kFlatThreads, stream, a, beside);
+            else launch_beside_block_kernel(ctx, defk::def_step_flat_kernel<false, kPolicy, false>, flat_grid, defk::kFlatThreads, stream, a, beside);
         });
         if (err != cudaSuccess) return cuda_fail(err, "def_step flat kernel launch");
         return DEF_OK;

@@ -439,12 +439,13 @@ def_step_block_kernel(const StepArgs a) {
 // floats with 16-byte accesses that ignore the row boundaries; every float finds its own
 // (worker, coordinate) and skips itself if the coordinate is in the block.  The block
 // coordinates -- exactly k of them -- are done beforehand by def_step_block_columns_kernel,
-// one thread per coordinate walking the W rows in order with 4-byte accesses.
+// one thread per coordinate walking the W rows in order with 4-byte accesses.  Both kernels
+// have a DETACH variant that also writes the next detach points z = x_{t+1} - lambda e'.
 // ---------------------------------------------------------------------------
 constexpr int kFlatThreads = 512;
 constexpr int64_t kFlatTile = (int64_t)kFlatThreads * 4;     // floats per CTA; needs n >= kFlatTile
 
-template <bool MOM, int U, int POL>
+template <bool MOM, int U, int POL, bool DETACH = false>
 __global__ void __launch_bounds__(256)
 def_step_block_columns_kernel(const StepArgs a) {
     // the flat kernel that follows touches no float of a block coordinate: let it start now
@@ -456,13 +457,13 @@ def_step_block_columns_kernel(const StepArgs a) {
     int64_t j = s + i;
     if (j >= a.d) j -= a.d;
     const int64_t col = j - a.j0;
-    if (col >= 0 && col < a.n) column_group<1, MOM, U, POL>(a, s, col);
+    if (col >= 0 && col < a.n) column_group<1, MOM, U, POL, DETACH>(a, s, col);
 }
 
 // The floats of one flat group of four, done one at a time: those that are not block coordinates
-// and lie inside the tensor.
-template <bool MOM>
-__device__ __forceinline__ void flat_group_by_floats(const StepArgs &a, int64_t f, int64_t total, const bool (&in)[4]) {
+// and lie inside the tensor.  c is the coordinate of float f (the group may run on into the next row).
+template <bool MOM, bool DETACH>
+__device__ __forceinline__ void flat_group_by_floats(const StepArgs &a, int64_t f, int64_t c, int64_t total, const bool (&in)[4]) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         if (in[i] || f + i >= total) continue;
@@ -475,7 +476,26 @@ __device__ __forceinline__ void flat_group_by_floats(const StepArgs &a, int64_t 
         worker_row<1, MOM>(g, m, e, no, a.eta, a.mu, true, m_new, e_new, u1);
         if (MOM) a.m[f + i] = m_new.v[0];
         a.e[f + i] = e_new.v[0];
+        if (DETACH) {                                     // not a block coordinate: x does not change in this step
+            int64_t ci = c + i;
+            if (ci >= a.n) ci -= a.n;
+            a.z[f + i] = __fmaf_rn(-a.lambda, e_new.v[0], a.x[ci]);
+        }
     }
+}
+
+// x at the four coordinates of a flat group that starts at coordinate c (it may run on into the
+// next row, i.e. wrap to coordinate 0): one 16-byte load where the group is aligned in x and whole.
+__device__ __forceinline__ Vec<4> flat_group_x(const StepArgs &a, int64_t c) {
+    Vec<4> x;
+    if ((c & 3) == 0 && c + 4 <= a.n) return load_vec<4, kCacheDefault>(a.x + c);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        int64_t ci = c + i;
+        if (ci >= a.n) ci -= a.n;
+        x.v[i] = a.x[ci];
+    }
+    return x;
 }
 
 // How many of the local coordinates [lo, hi) are block coordinates (runs A and B of touched_tiles,
@@ -500,19 +520,36 @@ __device__ __forceinline__ int64_t block_coordinates_in(const StepArgs &a, int64
 // per-thread bookkeeping), all of them (nothing to do), or mixed (every float checked).
 constexpr int kFlatPlain = 0, kFlatMixed = 1, kFlatIdle = 2;
 
-template <bool MOM, int POL>
+// With DETACH the kernel also writes z = x - lambda e' for its floats (x does not change outside the
+// block), which makes x a stream that every row reads.  The CTAs are then numbered so that x stays
+// in the L2: the coordinates are cut into segments of kFlatSegment; grid (W * a.chunk, segments);
+// CTA (r, seg) is the (r % a.chunk)-th of the flat CTAs whose first float lies in row r / a.chunk
+// within segment seg.  Every flat CTA's first float lies in exactly one (row, segment), so each
+// is done once; a (row, segment) holds a.chunk - 1 or a.chunk of them, the spare slot idles.
+constexpr int64_t kFlatSegment = (int64_t)1 << 20;            // coordinates: 4 MB of x and of every row
+
+template <bool MOM, int POL, bool DETACH = false>
 __global__ void __launch_bounds__(kFlatThreads)
 def_step_flat_kernel(const StepArgs a) {
-    __shared__ int64_t shared[3];
+    __shared__ int64_t shared[4];
     const int64_t total = (int64_t)a.W * a.n;                 // rows are contiguous: ld == n
-    const int64_t base = (int64_t)blockIdx.x * kFlatTile;
-    const int64_t f = base + (int64_t)threadIdx.x * 4;
     if (threadIdx.x == 0) {
+        int64_t cta = blockIdx.x;                             // which run of kFlatTile floats
+        int64_t kind = kFlatMixed;
+        if (DETACH) {
+            const int64_t w = (int64_t)blockIdx.x / a.chunk, i = (int64_t)blockIdx.x % a.chunk;
+            const int64_t c_lo = (int64_t)blockIdx.y * kFlatSegment;
+            const int64_t c_hi = c_lo + kFlatSegment < a.n ? c_lo + kFlatSegment : a.n;
+            const int64_t first = (w * a.n + c_lo + kFlatTile - 1) / kFlatTile;
+            const int64_t last = (w * a.n + c_hi + kFlatTile - 1) / kFlatTile;
+            cta = first + i;
+            if (cta >= last) kind = kFlatIdle;                // the spare slot of this (row, segment)
+        }
+        const int64_t base = cta * kFlatTile;
         const int64_t s = block_start(a.seed, a.step, a.d);
         const int64_t w0 = base / a.n;                        // worker of the CTA's first float
         const int64_t c0 = base - w0 * a.n;                   // and its coordinate
-        int64_t kind = kFlatMixed;
-        if (base + kFlatTile <= total) {                      // (the last, ragged CTA stays mixed)
+        if (kind != kFlatIdle && base + kFlatTile <= total) { // (the last, ragged CTA stays mixed)
             // the CTA's floats are coordinates [c0, c0 + kFlatTile) of one row, or -- n >= kFlatTile --
             // [c0, n) of one row and [0, c0 + kFlatTile - n) of the next
             const int64_t end = c0 + kFlatTile;
@@ -520,20 +557,32 @@ def_step_flat_kernel(const StepArgs a) {
             if (end > a.n) inside += block_coordinates_in(a, s, 0, end - a.n);
             kind = inside == 0 ? kFlatPlain : inside == kFlatTile ? kFlatIdle : kFlatMixed;
         }
-        shared[0] = s; shared[1] = c0; shared[2] = kind;
+        shared[0] = s; shared[1] = c0; shared[2] = kind; shared[3] = base;
     }
     __syncthreads();
     const int64_t kind = shared[2];
+    const int64_t f = shared[3] + (int64_t)threadIdx.x * 4;
     if (kind == kFlatPlain) {
         const bool none[4] = {false, false, false, false};
         float unused[4];
         const Vec<4> g = load_vec<4, POL>(a.g + f);
         const Vec<4> e = load_vec<4, POL>(a.e + f);
-        Vec<4> m, m_new, e_new;
+        Vec<4> m, m_new, e_new, x;
         if (MOM) m = load_vec<4, POL>(a.m + f);
+        if (DETACH) {
+            int64_t c = shared[1] + (int64_t)threadIdx.x * 4;
+            if (c >= a.n) c -= a.n;
+            x = flat_group_x(a, c);
+        }
         worker_row<4, MOM>(g, m, e, none, a.eta, a.mu, true, m_new, e_new, unused);
         if (MOM) store_vec<4, POL>(a.m + f, m_new);
         store_vec<4, POL>(a.e + f, e_new);
+        if (DETACH) {
+            Vec<4> z;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) z.v[i] = __fmaf_rn(-a.lambda, e_new.v[i], x.v[i]);
+            store_vec<4, POL>(a.z + f, z);
+        }
     } else if (kind == kFlatMixed && f < total) {
         const int64_t s = shared[0];
         int64_t c = shared[1] + (int64_t)threadIdx.x * 4;    // < 2 n because n >= kFlatTile
@@ -555,18 +604,25 @@ def_step_flat_kernel(const StepArgs a) {
             float unused[4];
             const Vec<4> g = load_vec<4, POL>(a.g + f);
             const Vec<4> e = load_vec<4, POL>(a.e + f);
-            Vec<4> m, m_new, e_new;
+            Vec<4> m, m_new, e_new, x;
             if (MOM) m = load_vec<4, POL>(a.m + f);
+            if (DETACH) x = flat_group_x(a, c);
             worker_row<4, MOM>(g, m, e, none, a.eta, a.mu, true, m_new, e_new, unused);
             if (MOM) store_vec<4, POL>(a.m + f, m_new);
             store_vec<4, POL>(a.e + f, e_new);
+            if (DETACH) {
+                Vec<4> z;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) z.v[i] = __fmaf_rn(-a.lambda, e_new.v[i], x.v[i]);
+                store_vec<4, POL>(a.z + f, z);
+            }
         } else if (!all) {
             // a group that straddles an edge of the block, or the last W * n % 4 floats: float by
             // float, touching nothing that is in the block (whose floats belong to the other kernel)
-            flat_group_by_floats<MOM>(a, f, total, in);
+            flat_group_by_floats<MOM, DETACH>(a, f, c, total, in);
         }
     }
-    if (blockIdx.x == 0 && threadIdx.x == 0) grid_dependency_wait();
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) grid_dependency_wait();
 }
 
 // Second half of a row-sharded step (Algorithm 1's update after the all-reduce):

@@ -710,6 +710,46 @@ def test_unaligned_contiguous_rows_take_the_flat_path(B, d):
     B.def_destroy(ctx)
 
 
+@pytest.mark.parametrize("d,momentum", [(5_000_001, 0.9), (3_000_002, 0.9), (2_100_003, 0.0), (2_051, 0.9)])
+def test_unaligned_rows_with_detach_take_the_flat_path(B, d, momentum):
+    """The step with the fused detach output on contiguous rows with d % 4 != 0: the flat stream in
+    its chunked order (several segments of coordinates, spare slots, ragged last CTA) and the
+    block-columns kernel, every element of x, e', m' and z against the oracle, wrapped blocks included."""
+    dev = torch.device("cuda")
+    W, k, seed, lam = 6, max(1, d // 16), 12, 0.3
+    rng = np.random.default_rng(d)
+    x, cx = guarded((d,), dev)
+    e, ce = guarded((W, d), dev); z, cz = guarded((W, d), dev)
+    x.copy_(torch.from_numpy((0.05 * rng.standard_normal(d)).astype(np.float32))); e.zero_(); z.fill_(-7.0)
+    m = cm = None
+    if momentum:
+        m, cm = guarded((W, d), dev); m.zero_()
+    xo = x.cpu().numpy().copy(); eo = np.zeros((W, d), np.float32)
+    mo = np.zeros((W, d), np.float32) if momentum else None
+    ctx = B.def_create(d, W, k, 0, 0.1, momentum, (lam, 0.0))
+    B.def_set_small_step_bytes(ctx, 0)
+    B.def_set_kernel_timing(ctx, True)
+    steps = [0, 1] + find_steps(d, k, seed, lambda s: s + k > d)[:1]
+    for t in steps:
+        gh = (0.1 * rng.standard_normal((W, d))).astype(np.float32)
+        g = torch.from_numpy(gh).to(dev)
+        B.def_step_detach(ctx, x, g, e, m, z, t, seed)
+        oracle.step(xo, gh, eo, mo, d=d, k=k, s=oracle.block_start(seed, t, d), eta=0.1, mu=momentum)
+        zh = z.cpu().numpy()
+        for w in range(W):
+            assert np.array_equal(zh[w], oracle.detach(xo, np.ascontiguousarray(eo[w]), lam)), (t, w)
+    assert B.def_kernel_time(ctx, B.DEF_KERNEL_STREAM)[1] == len(steps)
+    assert B.def_kernel_time(ctx, B.DEF_KERNEL_BLOCK)[1] == len(steps)
+    assert B.def_kernel_time(ctx, B.DEF_KERNEL_GENERAL)[1] == 0
+    assert np.array_equal(x.cpu().numpy(), xo) and np.array_equal(e.cpu().numpy(), eo)
+    if momentum:
+        assert np.array_equal(m.cpu().numpy(), mo)
+    for chk in (cx, ce, cz, cm):
+        if chk:
+            chk()
+    B.def_destroy(ctx)
+
+
 def test_random_shapes_and_layouts(B):
     """Seeded sweep over shapes, alignments, launch strategies, momentum on/off and the fused
     detach output: every case bit-identical to the oracle, nothing written outside the tensors."""

@@ -193,8 +193,8 @@ int def_set_rows_stream(def_ctx *ctx, void *side_stream);
 /*
  * One step with every tensor in HOST memory (pinned memory is much faster; pageable
  * works).  The library streams column ranges through device staging buffers it owns
- * (allocated on the first call, sized from the free device memory, freed by
- * def_destroy): host->device copy, def_step_columns' kernel and device->host copy of
+ * (allocated on the first call: three slots of up to 512 MiB of rows each, less for small
+ * models and when free device memory is short; freed by def_destroy): host->device copy, def_step_columns' kernel and device->host copy of
  * successive ranges overlap on three streams.  Blocks until params_host,
  * errors_host and mom_host hold the results.  Same shapes as def_step.
  */

@@ -259,7 +259,7 @@ def host_memory_available():
     return None
 
 
-def run_workload_every_element(B, wl, steps, check_at):
+def run_workload_every_element(B, wl, steps, check_at, detach=False):
     """Full-size run in the launch configuration the benchmark times, with the fp32 oracle stepping
     the WHOLE tensors beside it (its all-cores build: the same source and the same bits as the
     plain build, see test_oracle_parallel.py; no fp64 shadow at this size).  After the steps in
@@ -277,9 +277,13 @@ def run_workload_every_element(B, wl, steps, check_at):
     g_host = torch.empty(wl.W, wl.d, dtype=torch.float32).pin_memory()
     back = torch.empty(wl.W, wl.d, dtype=torch.float32).pin_memory()
     exact = True
+    z = torch.empty(wl.W, wl.d, dtype=torch.float32, device=dev) if detach else None
     for t in range(steps):
         WL.gradients(wl, t, dev, out=g, col_sigma=col_sigma)
-        B.def_step(ctx, x, g, e, m, t, wl.rbgs_seed)
+        if detach:
+            B.def_step_detach(ctx, x, g, e, m, z, t, wl.rbgs_seed)
+        else:
+            B.def_step(ctx, x, g, e, m, t, wl.rbgs_seed)
         g_host.copy_(g)
         s = o.block_start(wl.rbgs_seed, t, wl.d)
         assert B.def_block_start(ctx, t, wl.rbgs_seed) == s
@@ -289,9 +293,14 @@ def run_workload_every_element(B, wl, steps, check_at):
             for dev_t, host_t, name in ((e, eo, "errors"), (m, mo, "mom")):
                 back.copy_(dev_t)
                 exact &= compare(back.numpy(), host_t, "%s after %d steps" % (name, t + 1))
+            if detach:                                    # every worker's next detach point, every coordinate
+                back.copy_(z)
+                zh = back.numpy()
+                for w in range(wl.W):
+                    assert np.array_equal(zh[w], o.detach(xo, eo[w], wl.lam)), "detach point of worker %d" % w
     assert B.def_launch_count(ctx) == 2 * steps, "the kernel pair the benchmark times"
     B.def_destroy(ctx)
-    del g, e, m, x, g_host, back
+    del g, e, m, x, z, g_host, back
     torch.cuda.empty_cache()
     return exact
 
@@ -303,16 +312,28 @@ def test_config_full_size_every_element(B, cfg):
     assert run_workload_every_element(B, wl, wl.steps, {10, wl.steps})
 
 
-def test_config5_full_size_every_element(B):
-    """Config 5 (ratio 32, DEF) whole for its 10 steps: 2.2e9 elements per tensor.  The oracle's
-    state, its temporaries and the pinned staging buffers need about 60 GB of host memory."""
+def _config5_needs_host_memory():
     need = 80 << 30
     avail = host_memory_available()
     if avail is not None and avail < need:
-        pytest.skip("host has %.0f GB available; the whole-tensor run of config 5 needs about 60 GB "
-                    "(the sampled test covers this configuration)" % (avail / 2 ** 30))
-    wl = WL.get(5)
+        pytest.skip("host has %.0f GB available; a whole-tensor run of config 5 needs about 60 GB "
+                    "(the sampled tests cover this configuration)" % (avail / 2 ** 30))
+
+
+@pytest.mark.parametrize("ratio", [32, 8, 1000])
+def test_config5_full_size_every_element(B, ratio):
+    """Config 5 whole for its 10 steps at the default ratio and at both ends of its sweep: 2.2e9
+    elements per tensor.  The oracle's state, its temporaries and the pinned staging buffers need
+    about 60 GB of host memory."""
+    _config5_needs_host_memory()
+    wl = WL.get(5).with_ratio(ratio)
     assert run_workload_every_element(B, wl, wl.steps, {wl.steps})
+
+
+def test_config5_detach_output_every_element(B):
+    """Config 5 with the fused detach output, 3 steps: z of every worker on every coordinate."""
+    _config5_needs_host_memory()
+    assert run_workload_every_element(B, WL.get(5), 3, {3}, detach=True)
 
 
 def sample_columns(wl, steps, n_random=20000, halo=48):

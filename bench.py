@@ -730,10 +730,10 @@ def main():
             line["e2e"] = bench_rows_e2e(B, WL, wl, max(1, min(args.steps, 3)), 1, dist, world, rank)
             if world == 1:
                 line["cpu_baseline"] = cpu_baseline(wl, 20, 1)
-        if rank == 0:
-            print(json.dumps(line))
         if own_group or dist is not None:
             tdist.destroy_process_group()
+        if rank == 0:                                      # last, after whatever the communicator logs on its way out
+            print(json.dumps(line), flush=True)
         return
 
     small = wl.algorithmic_bytes_per_step() < 1e9          # fits the L2: flush it between steps
@@ -784,10 +784,10 @@ def main():
             line["per_config_note"] = ("EF, DEF and DEF-A run the same kernels given the gradients: the variant changes only "
                                        "where the caller evaluates them and the returned model")
             line["cpu_baseline"] = cpu_baseline(wl, 20, 1)
-    if rank == 0:
-        print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
+    if rank == 0:                                          # last, after whatever the communicator logs on its way out
+        print(json.dumps(line), flush=True)
 
 
 if __name__ == "__main__":

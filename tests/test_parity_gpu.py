@@ -493,8 +493,11 @@ def test_column_shards_on_the_kernel_pair(B, ratio):
     B.def_destroy(ctx)
 
 
+@pytest.mark.parametrize("pair", [False, True], ids=["general", "pair"])
 @pytest.mark.parametrize("momentum", [0.9, 0.0])
-def test_step_host_matches_oracle(B, momentum):
+def test_step_host_matches_oracle(B, momentum, pair):
+    """Every tensor in host memory, streamed through the staging slots in column pieces; with `pair`
+    every piece runs the kernel pair on its column range (as the pieces of a large model do)."""
     wl = WL.get(1).scaled(3_000_001, W=5, momentum=momentum)      # odd d: unaligned host rows
     d, W, k = wl.d, wl.W, wl.k
     x = WL.initial_params(wl, "cpu").pin_memory()
@@ -503,6 +506,8 @@ def test_step_host_matches_oracle(B, momentum):
     xo = x.numpy().copy(); eo = np.zeros((W, d), np.float32)
     mo = np.zeros((W, d), np.float32) if momentum else None
     ctx = B.def_create(d, W, k, wl.variant, wl.lr, momentum)
+    if pair:
+        B.def_set_small_step_bytes(ctx, 0)
     for t in range(3):
         g = WL.gradients(wl, t, "cpu").pin_memory()
         B.def_step_host(ctx, x, g, e, m, t, 4)

@@ -795,3 +795,55 @@ def test_random_shapes_and_layouts(B):
             run_detach(B, d, W, k, steps, momentum, float(rng.choice([0.0, 0.3, 1.0])), offsets=offsets, seed=seed, pair=pair)
         else:
             assert run_whole(B, d, W, k, steps, momentum, seed, offsets=offsets[:4], pair=pair), (case, d, W, k)
+
+
+def test_random_column_views(B):
+    """Seeded sweep over column ranges of larger models (any j0 and n, padded or contiguous rows),
+    block lengths from 1 to d, both launch strategies, momentum on / off and the fused detach
+    output: every case bit-identical to the oracle's column view, padding columns untouched."""
+    dev = torch.device("cuda")
+    rng = np.random.default_rng(20261130)
+    for case in range(250):
+        d = int(rng.choice([rng.integers(2048, 20000), rng.integers(20000, 400000)]))
+        W = int(rng.choice([1, 2, 3, 5, 8, 16]))
+        k = int(rng.choice([1, d, d - 1, max(1, d // 2), max(1, d // 8), int(rng.integers(1, d + 1))]))
+        mom = float(rng.choice([0.0, 0.9]))
+        detach = bool(rng.integers(0, 2))
+        lam, seed = 0.3, int(rng.integers(0, 1000))
+        if rng.random() < 0.5:
+            j0, n = 0, d
+        else:
+            j0 = int(rng.integers(0, d)); n = int(rng.integers(1, d - j0 + 1))
+            if rng.random() < 0.5:
+                j0 = j0 // 4 * 4
+        ld = n if rng.random() < 0.5 else (n + 3) // 4 * 4 + int(rng.choice([0, 4]))
+        x0 = (0.05 * rng.standard_normal(d)).astype(np.float32)
+        cols = np.arange(j0, j0 + n, dtype=np.int64)
+        xo = x0[j0:j0 + n].copy(); eo = np.zeros((W, n), np.float32)
+        mo = np.zeros((W, n), np.float32) if mom else None
+        x = torch.from_numpy(xo.copy()).to(dev)
+        e = torch.zeros(W, ld, device=dev); m = torch.zeros(W, ld, device=dev) if mom else None
+        z = torch.full((W, ld), -9.0, device=dev) if detach else None
+        ctx = B.def_create(d, W, k, 0, 0.1, mom, (lam, 0.0))
+        B.def_set_small_step_bytes(ctx, 0 if rng.random() < 0.8 else 1 << 60)
+        what = dict(case=case, d=d, W=W, k=k, mom=mom, detach=detach, j0=j0, n=n, ld=ld, seed=seed)
+        for t in (int(v) for v in rng.integers(0, 10 ** 6, size=3)):
+            gh = (0.1 * rng.standard_normal((W, n))).astype(np.float32)
+            g = torch.zeros(W, ld, device=dev); g[:, :n] = torch.from_numpy(gh).to(dev)
+            if detach:
+                B.def_step_columns_detach(ctx, j0, n, ld, x, g, e, m, z, t, seed)
+            else:
+                B.def_step_columns(ctx, j0, n, ld, x, g, e, m, t, seed)
+            oracle.step(xo, gh, eo, mo, d=d, k=k, s=oracle.block_start(seed, t, d), eta=0.1, mu=mom,
+                        cols=cols if n != d else None)
+            if detach:
+                zh = z[:, :n].cpu().numpy()
+                for w in range(W):
+                    assert np.array_equal(zh[w], oracle.detach(xo, np.ascontiguousarray(eo[w]), lam)), (what, t, w)
+        assert np.array_equal(x.cpu().numpy(), xo) and np.array_equal(e[:, :n].cpu().numpy(), eo), what
+        if mom:
+            assert np.array_equal(m[:, :n].cpu().numpy(), mo), what
+        assert not e[:, n:].any(), what
+        if detach:
+            assert bool((z[:, n:] == -9.0).all()), what
+        B.def_destroy(ctx)

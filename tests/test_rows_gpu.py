@@ -196,3 +196,47 @@ def test_rows_argument_checks(B):
     assert B.lib.def_set_stream(ctx.handle, s.cuda_stream) == B.DEF_ERR_ARG
     B.def_set_rows_stream(ctx, None)
     B.def_destroy(ctx)
+
+
+def test_random_shapes_rows_halves_equal_def_step(B):
+    """Seeded sweep: the two halves of the row-sharded step with all workers on one rank (no
+    collective between them) against def_step / def_step_detach -- any d, k from 1 to d, both launch
+    strategies, with and without momentum, the detach output and the side stream -- bit for bit,
+    with nothing between the calls that waits for the GPU."""
+    dev = torch.device("cuda", 0)
+    rng = np.random.default_rng(20261201)
+    side = torch.cuda.Stream()
+    for case in range(150):
+        d = int(rng.choice([rng.integers(1, 3000), rng.integers(3000, 300000)]))
+        W = int(rng.choice([1, 2, 3, 5, 8]))
+        k = int(rng.choice([1, d, max(1, d - 1), max(1, d // 2), int(rng.integers(1, d + 1))]))
+        mom = float(rng.choice([0.0, 0.9])); detach = bool(rng.integers(0, 2)); use_side = bool(rng.integers(0, 2))
+        pair = 0 if rng.random() < 0.8 else 1 << 60
+        what = dict(case=case, d=d, W=W, k=k, mom=mom, detach=detach, side=use_side, pair=pair)
+        ctx1 = B.def_create(d, W, k, 0, 0.1, mom, (0.4, 0.0)); ctx2 = B.def_create(d, W, k, 0, 0.1, mom, (0.4, 0.0))
+        B.def_set_small_step_bytes(ctx1, pair); B.def_set_small_step_bytes(ctx2, pair)
+        if use_side:
+            B.def_set_rows_stream(ctx2, side)
+        x1 = torch.randn(d, device=dev) * 0.05; x2 = x1.clone()
+        e1 = torch.zeros(W, d, device=dev); e2 = torch.zeros(W, d, device=dev)
+        m1 = torch.zeros(W, d, device=dev) if mom else None; m2 = torch.zeros(W, d, device=dev) if mom else None
+        z1 = torch.full((W, d), -1.0, device=dev); z2 = torch.full((W, d), -2.0, device=dev)
+        blk = torch.full((k,), 5.0, device=dev)
+        gs = [torch.randn(W, d, device=dev) * 0.1 for _ in range(4)]
+        torch.cuda.synchronize()
+        for t, g in zip((int(v) for v in rng.integers(0, 10 ** 6, size=4)), gs):
+            if detach:
+                B.def_step_detach(ctx1, x1, g, e1, m1, z1, t, 3)
+                B.def_step_rows_local_detach(ctx2, x2, g, e2, m2, blk, z2, t, 3)
+                B.def_step_rows_apply_detach(ctx2, x2, blk, W, z2, t, 3)
+            else:
+                B.def_step(ctx1, x1, g, e1, m1, t, 3)
+                B.def_step_rows_local(ctx2, g, e2, m2, blk, t, 3)
+                B.def_step_rows_apply(ctx2, x2, blk, W, t, 3)
+        torch.cuda.synchronize()
+        assert torch.equal(x1, x2) and torch.equal(e1, e2), what
+        assert not mom or torch.equal(m1, m2), what
+        assert not detach or torch.equal(z1, z2), what
+        if use_side:
+            B.def_set_rows_stream(ctx2, None)
+        B.def_destroy(ctx1); B.def_destroy(ctx2)
